@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the Thanos per-layer hot path on B200.
+
+A "step" is one pass of the whole hot path over one transformer block's layer set: for every
+distinct layer input the calibration Hessian (thanos_hessian_accumulate over all tokens) and
+its factorisation (thanos_prepare_inverse), then thanos_prune_layer for every layer.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the float64 CPU oracle on a bounded
+sample of the same workload instead.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import workloads as WL
+
+METRIC = "pruned_weights_per_sec"
+UNIT = "weights/s"
+TOKEN_CHUNK = 32768  # tokens per thanos_hessian_accumulate call
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def layer_set_weights(cfg):
+    return sum(L.c * L.b for L in cfg.layers)
+
+
+def mode_args(cfg, T):
+    if cfg.mode == "unstructured":
+        return dict(mode=T.UNSTRUCTURED, p=cfg.p)
+    return dict(mode=T.NM, n=cfg.n, m=cfg.m)
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch.distributed as dist
+
+    import paper_2504_05346_b200 as T
+    from paper_2504_05346_b200 import build as B_
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        B_.build()
+    if world > 1:
+        dist.barrier()
+    T.load_library()
+
+    cfg = WL.CONFIGS[args.workload]
+    a = args.tokens or cfg.a
+    dt = T.BF16 if cfg.dtype == "bf16" else T.F32
+    margs = mode_args(cfg, T)
+
+    # ---- resident inputs: one activation matrix per distinct layer input, all weights
+    inputs = {}
+    for L in cfg.layers:
+        if L.input_id not in inputs:
+            inputs[L.input_id] = WL.config_activations(cfg, L.input_id, L.b, device=dev, a=a)
+    weights = [WL.config_weight(cfg, i, device=dev) for i in range(len(cfg.layers))]
+    outs = [torch.empty_like(w) for w in weights]
+    masks = [torch.empty(w.shape, dtype=torch.uint8, device=dev) for w in weights]
+    bs = sorted({L.b for L in cfg.layers})
+    Hbuf = {b: torch.empty((b, b), dtype=torch.float32, device=dev) for b in bs}
+    ws_bytes = 256
+    for L in cfg.layers:
+        ws_bytes = max(ws_bytes, T.workspace_bytes(0, 0, L.b, 0, dt),
+                       T.workspace_bytes(1, 0, L.b, 0, T.F32),
+                       T.workspace_bytes(2, L.c, L.b, cfg.B, dt))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    hess_events = []  # (start, end, flops) per thanos_hessian_accumulate call
+    phase_events = {"hessian": [], "prepare": [], "prune": []}
+
+    def one_step(record):
+        stats_all = []
+        for iid, X in inputs.items():
+            b = X.shape[1]
+            H = Hbuf[b]
+            e0 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            H.zero_()
+            for t0 in range(0, a, TOKEN_CHUNK):
+                xc = X[t0:t0 + TOKEN_CHUNK]
+                if record:
+                    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    s.record()
+                T.hessian_accumulate(H, xc, workspace=ws)
+                if record:
+                    e.record()
+                    hess_events.append((s, e, float(xc.shape[0]) * b * (b + 1)))
+            e1 = torch.cuda.Event(enable_timing=True)
+            e1.record()
+            U, xn = T.prepare_inverse(H, cfg.damp_rel, workspace=ws, check=False)
+            e2 = torch.cuda.Event(enable_timing=True)
+            e2.record()
+            for i, L in enumerate(cfg.layers):
+                if L.input_id != iid:
+                    continue
+                _, _, st = T.prune_layer(weights[i], U, xn, B=cfg.B, workspace=ws, out=outs[i],
+                                         mask=masks[i], read_stats=False, **margs)
+                stats_all.append(st)
+            e3 = torch.cuda.Event(enable_timing=True)
+            e3.record()
+            if record:
+                phase_events["hessian"].append((e0, e1))
+                phase_events["prepare"].append((e1, e2))
+                phase_events["prune"].append((e2, e3))
+            del U, xn
+        return stats_all
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step(False)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = T.launch_count()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_start.record()
+    stats_last = None
+    for _ in range(args.steps):
+        stats_last = one_step(True)
+    t_end.record()
+    barrier()
+    launches = T.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t_start.elapsed_time(t_end)
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    # device status of the last step
+    for st in stats_last:
+        ps = T.PruneStats.from_bytes(bytes(st.cpu().numpy().tobytes()))
+        if ps.status != 0:
+            raise RuntimeError("device status %d in prune_layer" % ps.status)
+
+    nweights = layer_set_weights(cfg)
+    ms_per_step = ms_total / args.steps
+    value = world * nweights * args.steps / (ms_total * 1e-3)
+
+    # ---- roofline of the dominant kernel: the Hessian contraction
+    peaks = _peaks()
+    h_ms = sum(s.elapsed_time(e) for s, e, _ in hess_events)
+    h_flops = sum(f for _, _, f in hess_events)
+    achieved = h_flops / (h_ms * 1e-3) / 1e12 if h_ms > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    phase_ms = {k: sum(s.elapsed_time(e) for s, e in v) / args.steps for k, v in phase_events.items()}
+    roofline = {"kernel": "hessian_accumulate", "bound": "tensor", "achieved": round(achieved, 2),
+                "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
+                "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None,
+                "launches": len(hess_events), "avg_launch_ms": round(h_ms / max(1, len(hess_events)), 4)}
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(T, cfg, a, dev, dt, margs, world, args)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample(cfg, args.cpu_budget_s)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype if cfg.dtype != "f32" else "f32",
+            "data": "synthetic",
+            "config": {"workload": "%s layer set: %s; %d calibration tokens; %s; B=%d; damp %.2g"
+                                   % (cfg.name, ", ".join("%dx%d" % (L.c, L.b) for L in cfg.layers),
+                                      a, ("%d%% unstructured" % round(100 * cfg.p))
+                                      if cfg.mode == "unstructured" else "%d:%d" % (cfg.n, cfg.m),
+                                      cfg.B, cfg.damp_rel),
+                       "weights_per_step": nweights, "l2": "inputs larger than L2",
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "token_chunk": TOKEN_CHUNK},
+            "ms_per_layer": ms_per_step / len(cfg.layers),
+            "phase_ms_per_step": {k: round(v, 3) for k, v in phase_ms.items()},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(T, cfg, a, dev, dt, margs, world, args):
+    """Same metric through thanos_prune_layer_host: pinned host inputs, copies timed."""
+    import torch.distributed as dist
+
+    steps = max(1, min(args.steps, args.e2e_steps))
+    host_in = {}
+    for L in cfg.layers:
+        if L.input_id not in host_in:
+            x = WL.config_activations(cfg, L.input_id, L.b, device=dev, a=a)
+            host_in[L.input_id] = x.cpu().pin_memory()
+            del x
+    host_w = [WL.config_weight(cfg, i, device=dev).cpu().pin_memory() for i in range(len(cfg.layers))]
+    host_o = [torch.empty_like(w).pin_memory() for w in host_w]
+    host_m = [torch.empty(w.shape, dtype=torch.uint8).pin_memory() for w in host_w]
+    torch.cuda.empty_cache()
+    arena_bytes = max(T.workspace_bytes(3, L.c, L.b, cfg.B, dt) for L in cfg.layers)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
+    h2d = sum(x.numel() * x.element_size() for x in host_in.values()) + \
+        sum(w.numel() * w.element_size() for w in host_w)
+    d2h = sum(w.numel() * w.element_size() + w.numel() + 64 for w in host_w)
+
+    def step():
+        seen = None
+        order = sorted(range(len(cfg.layers)), key=lambda i: cfg.layers[i].input_id)
+        for i in order:
+            L = cfg.layers[i]
+            reuse = seen == L.input_id
+            T.prune_layer_host(host_w[i], None if reuse else host_in[L.input_id], cfg.damp_rel,
+                               B=cfg.B, arena=arena, reuse_factor=reuse, out=host_o[i],
+                               mask=host_m[i], **margs)
+            seen = L.input_id
+
+    step()  # warm-up
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt_s = time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([dt_s], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt_s = float(tt.item())
+    return {"value": world * layer_set_weights(cfg) * steps / dt_s, "unit": UNIT,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
+            "ms_per_step": dt_s * 1e3 / steps}
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample(cfg, budget_s=20.0):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: the first
+    layer of the set with a reduced token count and only the first column blocks of the sweep;
+    the per-weight rate is extrapolated to the full layer (stated in `sample`)."""
+    from oracle import thanos_oracle as O
+
+    try:
+        import threadpoolctl
+        info = threadpoolctl.threadpool_info()
+        cores = max([i.get("num_threads", 1) for i in info] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    L = cfg.layers[0]
+    c, b, B = L.c, L.b, cfg.B
+    a_s = min(cfg.a, 4096)
+    W = WL.config_weight(cfg, 0).double().numpy()
+    Xt = WL.config_activations(cfg, L.input_id, b, a=a_s).double().numpy()
+    t0 = time.perf_counter()
+    H = O.hessian(Xt.T)
+    t_h = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    Hd = O.damped(H, cfg.damp_rel)
+    U = O.inverse_factor(Hd)
+    xn = O.feature_norms(H)
+    t_f = time.perf_counter() - t0
+    # sweep: as many leading blocks as fit the budget (at least one)
+    Wc = W.copy()
+    r = int(np.floor(cfg.p * c * b)) if cfg.mode == "unstructured" else 0
+    nblk_total = -(-b // B)
+    t_sweep, nblk = 0.0, 0
+    for j1 in range(0, b, B):
+        t0 = time.perf_counter()
+        j2 = min(b, j1 + B)
+        if cfg.mode == "unstructured":
+            Mb = O.psi(Wc[:, j1:], xn[j1:], r)[:, : j2 - j1]
+            r -= int(Mb.sum())
+        else:
+            Mb = O.nm_block_mask(Wc[:, j1:j2], xn[j1:j2], cfg.n, cfg.m)
+        O.block_update_from_factor(Wc, Mb, U, j1, j2)
+        t_sweep += time.perf_counter() - t0
+        nblk += 1
+        if t_h + t_f + t_sweep > budget_s:
+            break
+    t_full = t_h * (cfg.a / a_s) + t_f + t_sweep * (nblk_total / nblk)
+    return {"value": c * b / t_full, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": "layer %dx%d: Hessian on %d of %d tokens (%.1fs, scaled by token count), "
+                      "factor (%.1fs), first %d of %d column blocks of the sweep (%.1fs, scaled by "
+                      "block count)" % (c, b, a_s, cfg.a, t_h, t_f, nblk, nblk_total, t_sweep),
+            "seconds_measured": round(t_h + t_f + t_sweep, 2),
+            "seconds_extrapolated_layer": round(t_full, 1)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = WL.CONFIGS[args.workload]
+    vals, last = [], None
+    t0 = time.perf_counter()
+    for i in range(args.warmup + args.steps):
+        last = oracle_sample(cfg, budget_s=min(args.cpu_budget_s, 12.0))
+        if i >= args.warmup:
+            vals.append(last["value"])
+        if time.perf_counter() - t0 > 240 and vals:
+            break
+    value = float(np.mean(vals))
+    nweights = cfg.layers[0].c * cfg.layers[0].b
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": len(vals),
+            "warmup": args.warmup, "ms_per_step": 1e3 * nweights / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": "%s (float64 CPU oracle on a bounded sample, extrapolated)"
+                                   % cfg.name},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"],
+                             "kind": "oracle", "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b", choices=sorted(WL.CONFIGS))
+    ap.add_argument("--tokens", type=int, default=0, help="override the calibration token count")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,193 @@
+/*
+ * thanos.h -- C ABI of the B200 (sm_100a) library for the per-layer hot path of the Thanos
+ * block-wise pruning method (arXiv 2504.05346).
+ *
+ * Notation follows the paper's notation table: a linear layer has weights W (c x b; c output
+ * features = rows, b input features = columns), calibration inputs X (b x a; a tokens), the
+ * Hessian H = 2 X X^T (b x b), block width B, sparsity ratio p, and a mask M with
+ * M_ij = 1 meaning "weight W_ij is removed" (Section 2.1).
+ *
+ * Conventions shared by every call
+ *  - All data pointers are DEVICE pointers unless the argument is documented as "host".
+ *  - The caller owns every buffer.  The library allocates no device memory and keeps no
+ *    global state between calls (except the entry point documented otherwise at the end of
+ *    this header); scratch space is the caller-provided `workspace` whose minimum size
+ *    comes from thanos_workspace_bytes().
+ *  - Matrices are row-major and dense (leading dimension = number of columns) unless a
+ *    leading dimension argument is present.
+ *  - Calls are asynchronous: work is enqueued on `stream` (a cudaStream_t passed as
+ *    void*; NULL is the legacy default stream) and the call returns without waiting.
+ *  - Errors detectable on the host (null pointers, bad shapes, misalignment, workspace too
+ *    small) are returned immediately and nothing is launched.  Conditions only the device
+ *    can see (a non-positive Cholesky pivot, a bounded wait that ran out) are written to a
+ *    status word in device memory (first error wins); the caller reads it after
+ *    synchronising the stream.  Outputs are unspecified after an error.
+ *  - Every pointer must be 16-byte aligned.
+ */
+#ifndef THANOS_H_
+#define THANOS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  THANOS_OK = 0,
+  THANOS_ERR_INVALID_ARG = 1, /* null pointer, value out of range                         */
+  THANOS_ERR_SHAPE = 2,       /* a dimension violates a documented constraint              */
+  THANOS_ERR_DTYPE = 3,       /* unknown thanos_dtype_t                                    */
+  THANOS_ERR_ALIGNMENT = 4,   /* pointer or leading dimension not aligned as documented    */
+  THANOS_ERR_WORKSPACE = 5,   /* workspace missing or smaller than thanos_workspace_bytes */
+  THANOS_ERR_NOT_SPD = 6,     /* a Cholesky pivot was <= 0 or not finite (device status)   */
+  THANOS_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (device status)        */
+  THANOS_ERR_CUDA = 8         /* a CUDA runtime / driver call failed                       */
+} thanos_status_t;
+
+typedef enum { THANOS_F32 = 0, THANOS_BF16 = 1 } thanos_dtype_t;
+typedef enum { THANOS_UNSTRUCTURED = 0, THANOS_NM = 1 } thanos_mode_t;
+
+/* Which call a workspace query refers to. */
+typedef enum {
+  THANOS_WS_HESSIAN = 0,
+  THANOS_WS_PREPARE = 1,
+  THANOS_WS_PRUNE = 2,
+  THANOS_WS_HOST_LAYER = 3
+} thanos_ws_which_t;
+
+/* Per-call statistics and device-side status of thanos_prune_layer / thanos_prune_block,
+ * written to device memory (64 bytes). */
+typedef struct {
+  int32_t status;       /* thanos_status_t of the first device-detected error, 0 if none  */
+  int32_t err_index;    /* row (solve) or column (factorisation) where it was detected    */
+  int64_t n_pruned;     /* number of mask entries set to 1 so far                          */
+  int64_t r_left;       /* unstructured: removals still to place after the last block run */
+  int32_t max_s;        /* largest per-row system size s seen                              */
+  int32_t n_blocks;     /* column blocks processed                                         */
+  int64_t n_tied;       /* unstructured: entries whose metric equals a block threshold
+                           bit-for-bit but which the (row, column) tie-break left unpruned */
+  uint32_t last_threshold_bits; /* fp32 bit pattern of the last block's threshold metric  */
+  int32_t reserved[5];
+} thanos_stats_t;
+
+/*
+ * Hessian accumulation: H += 2 * X_chunk^T X_chunk   (Section 3.2: H = 2 X X^T; summing over
+ * calibration chunks is the un-averaged d-sample Hessian of Appendix A.4).
+ *
+ *  H       device, fp32 [b, b], full symmetric storage; the caller zeroes it before the first
+ *          chunk.  Updated in place; stays exactly symmetric.
+ *  X       device, [n_tok, b] tokens-major (the transpose of the paper's X), element type
+ *          `xdtype`, leading dimension `ldx` elements (ldx >= b, ldx % 8 == 0).
+ *  b % 8 == 0, n_tok >= 0 (0 is a no-op).
+ *  workspace: thanos_workspace_bytes(THANOS_WS_HESSIAN, 0, b, 0, xdtype) bytes.
+ * May be called any number of times; the order of floating-point summation across a call's
+ * internal token slices is not fixed, so results can differ in the last bits between runs.
+ */
+thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X,
+                                          thanos_dtype_t xdtype, int64_t n_tok, int64_t ldx,
+                                          void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Factor the damped Hessian so that the inverse of every trailing block is available
+ * (Algorithm 1, last line of the block loop: the Hessian is restricted to the unseen columns
+ * and re-inverted for every block; Appendix F.7 counts that as O(b^4 / B)).  This call
+ * replaces all those inversions by one factorisation:
+ *
+ *   H_d = H + damp_rel * mean(diag H) * I          (damping as in Algorithm 5, line 3)
+ *   factor = upper-triangular U with U^T U = H_d^{-1}; then for every j
+ *   inv(H_d[j:, j:]) = U[j:, j:]^T U[j:, j:].
+ *   xnorm[j] = sqrt(H_jj / 2) = ||X_j:||_2 from the UNDAMPED diagonal (metric of Eq. 4).
+ *
+ *  H        device, fp32 [b, b], read only (only the upper triangle is read).
+ *  factor   device, fp32 [b, b]; entries below the diagonal are written as 0.
+ *  xnorm    device, fp32 [b].
+ *  status_dev device int32[2]: {thanos_status_t, failing column}; the caller zeroes it.
+ *  workspace: thanos_workspace_bytes(THANOS_WS_PREPARE, 0, b, 0, THANOS_F32) bytes.
+ * damp_rel >= 0; with damp_rel = 0 a singular H is reported as THANOS_ERR_NOT_SPD.
+ */
+thanos_status_t thanos_prepare_inverse(const float* H, int64_t b, float damp_rel, float* factor,
+                                       float* xnorm, void* workspace, size_t ws_bytes,
+                                       int32_t* status_dev, void* stream);
+
+/*
+ * Prune one layer: the block sweep of Algorithm 1 (mode THANOS_UNSTRUCTURED) or of
+ * Algorithm 4 with alpha = 0 (mode THANOS_NM).  For each block of B columns, left to right:
+ * metric |W_ij| * xnorm_j on the current weights (Section 4.2), block mask (Eq. psi over the
+ * whole residual with running budget r = floor(p c b), or the n smallest of every aligned
+ * group of m columns per row), per-row system lambda-hat R-hat = u and update
+ * W_{i, j1:b} <- w - u R-hat^{-1} R (Eqs. 5-8), removed entries set to exact 0.
+ *
+ *  W_in     device [c, b], element type wdtype.
+ *  W_out    device [c, b], same type; may alias W_in.
+ *  mask_out device uint8 [c, b]; 1 = removed.
+ *  factor, xnorm: outputs of thanos_prepare_inverse for this layer's input.
+ *  mode UNSTRUCTURED: 0 <= p < 1 (n, m ignored).  Metric ties are broken by (row, column)
+ *  ascending.  mode NM: 0 < n < m <= 32, B % m == 0, b % m == 0; n weights are REMOVED per
+ *  group; ties by column ascending.
+ *  1 <= B <= 512, B % 8 == 0, b % 8 == 0.  Per-row systems up to s = 320 unknowns are
+ *  supported (s <= B; s = n B / m in NM mode); larger -> THANOS_ERR_SHAPE.
+ *  stats_dev device thanos_stats_t, zeroed by this call.
+ *  workspace: thanos_workspace_bytes(THANOS_WS_PRUNE, c, b, B, wdtype) bytes.
+ */
+thanos_status_t thanos_prune_layer(const void* W_in, void* W_out, uint8_t* mask_out,
+                                   thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                   const float* factor, const float* xnorm, thanos_mode_t mode,
+                                   double p, int32_t n, int32_t m, int32_t B, void* workspace,
+                                   size_t ws_bytes, thanos_stats_t* stats_dev, void* stream);
+
+/*
+ * One block step of the sweep from a caller-supplied state (the body of the block loop of
+ * Algorithm 1 / Algorithm 4), for step-by-step checking against a reference.
+ *
+ *  Wc       device fp32 [c, b] working weights, updated in place for columns >= j1.
+ *  mask     device uint8 [c, b]; columns [j1, min(b, j1+B)) are written.
+ *  r_dev    device int64: removals still to place (unstructured); read and decremented by the
+ *           number of entries this block removed.  Ignored in NM mode (may be NULL).
+ *  stats_dev is accumulated into, not zeroed.
+ *  j1 % B == 0.  Same workspace as thanos_prune_layer.
+ */
+thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t b,
+                                   const float* factor, const float* xnorm, thanos_mode_t mode,
+                                   int32_t n, int32_t m, int32_t B, int64_t j1, int64_t* r_dev,
+                                   void* workspace, size_t ws_bytes, thanos_stats_t* stats_dev,
+                                   void* stream);
+
+/*
+ * The whole path for one layer from HOST buffers: copies X (in token chunks) and W to the
+ * device, runs thanos_hessian_accumulate, thanos_prepare_inverse and thanos_prune_layer, and
+ * copies W_pruned, the mask and the statistics back.  Synchronises `stream` before returning.
+ *
+ *  W_in_host, X_host, W_out_host, mask_out_host, stats_host: HOST pointers (pinned memory
+ *  gives the best copy rate; pageable works).  X_host is [a, b] tokens-major.
+ *  arena: DEVICE scratch of thanos_workspace_bytes(THANOS_WS_HOST_LAYER, c, b, B, dtype) bytes
+ *  holding H, the factor, the staged inputs and the per-call workspaces.
+ *  If reuse_factor != 0 the Hessian and factor left in `arena` by the previous call with the
+ *  same b are reused and X_host is not read (layers that share an input, e.g. q/k/v).
+ */
+thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_host,
+                                        void* W_out_host, uint8_t* mask_out_host,
+                                        thanos_dtype_t dtype, int64_t c, int64_t b, int64_t a,
+                                        float damp_rel, thanos_mode_t mode, double p, int32_t n,
+                                        int32_t m, int32_t B, int32_t reuse_factor, void* arena,
+                                        size_t arena_bytes, thanos_stats_t* stats_host,
+                                        void* stream);
+
+/* Minimum workspace in bytes for a call (see thanos_ws_which_t); 0 for unsupported shapes. */
+size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
+
+/* Static, NUL-terminated description of a status code. */
+const char* thanos_status_string(thanos_status_t status);
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+int32_t thanos_version(void);
+
+/* Number of kernels this library has launched in the calling process since it was loaded
+ * (host counter, for benchmarks that report launch counts). */
+int64_t thanos_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* THANOS_H_ */

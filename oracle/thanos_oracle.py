@@ -251,6 +251,24 @@ def inverse_factor(Hd: np.ndarray) -> np.ndarray:
     return np.linalg.cholesky(Hinv).T
 
 
+def block_update_from_factor(Wc, Mb, U, j1, j2):
+    """One block of the sweep (in place on ``Wc[:, j1:]``) with the residual inverse rows
+    rebuilt from the factor ``U``: Eqs. 5-8 for every row, removed entries set to 0."""
+    c = Wc.shape[0]
+    Ubb = U[j1:j2, j1:j2]
+    P = Ubb.T @ U[j1:j2, j1:]  # rows j1..j2 of inv(Hd[j1:, j1:])
+    G = P[:, : j2 - j1]
+    Lam = np.zeros((c, j2 - j1), dtype=F64)
+    for i in range(c):
+        q = phi(Mb[i])
+        if q.size == 0:
+            continue
+        Lam[i, q] = np.linalg.solve(G[np.ix_(q, q)].T, Wc[i, j1 + q])
+    Wc[:, j1:] -= Lam @ P
+    blk = Wc[:, j1:j2]
+    blk[Mb.astype(bool)] = 0.0
+
+
 def _sweep_fast(W, H, xnorm, B, damp_rel, block_mask_fn):
     W = np.asarray(W, dtype=F64)
     c, b = W.shape
@@ -260,18 +278,7 @@ def _sweep_fast(W, H, xnorm, B, damp_rel, block_mask_fn):
     for j1 in range(0, b, B):
         j2 = min(b, j1 + B)
         Mb = block_mask_fn(Wc, j1, j2)
-        Ubb = U[j1:j2, j1:j2]
-        P = Ubb.T @ U[j1:j2, j1:]  # rows j1..j2 of inv(Hd[j1:, j1:])
-        G = P[:, : j2 - j1]
-        Lam = np.zeros((c, j2 - j1), dtype=F64)
-        for i in range(c):
-            q = phi(Mb[i])
-            if q.size == 0:
-                continue
-            Lam[i, q] = np.linalg.solve(G[np.ix_(q, q)].T, Wc[i, j1 + q])
-        Wc[:, j1:] -= Lam @ P
-        blk = Wc[:, j1:j2]
-        blk[Mb.astype(bool)] = 0.0
+        block_update_from_factor(Wc, Mb, U, j1, j2)
         M[:, j1:j2] = Mb
     return Wc, M
 

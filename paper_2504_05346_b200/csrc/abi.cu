@@ -1,0 +1,267 @@
+// extern "C" entry points: argument checks, workspace carving, dispatch.
+#include "common.cuh"
+
+namespace thanos {
+
+std::atomic<long long> g_launch_count{0};
+
+thanos_status_t hessian_accumulate_simt(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
+                                        int64_t n_tok, int64_t ldx, cudaStream_t stream);
+size_t hessian_workspace_bytes(int64_t b, thanos_dtype_t dtype);
+thanos_status_t hessian_accumulate_impl(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
+                                        int64_t n_tok, int64_t ldx, void* workspace,
+                                        size_t ws_bytes, cudaStream_t stream);
+size_t prepare_workspace_bytes(int64_t b);
+thanos_status_t prepare_inverse_impl(const float* H, int64_t b, float damp_rel, float* factor,
+                                     float* xnorm, void* workspace, size_t ws_bytes,
+                                     int32_t* status_dev, cudaStream_t stream);
+size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
+thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, double p, int32_t n,
+                                    int32_t m, int32_t B);
+thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b, const float* U,
+                                 const float* xnorm, thanos_mode_t mode, int32_t n, int32_t m,
+                                 int32_t B, int64_t j1, int64_t* r_dev, void* workspace,
+                                 size_t ws_bytes, thanos_stats_t* stats, cudaStream_t stream);
+thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+                                 thanos_dtype_t wdtype, int64_t c, int64_t b, const float* U,
+                                 const float* xnorm, thanos_mode_t mode, double p, int32_t n,
+                                 int32_t m, int32_t B, void* workspace, size_t ws_bytes,
+                                 thanos_stats_t* stats, cudaStream_t stream);
+
+namespace {
+
+constexpr int64_t MAX_B = 65536;
+constexpr int64_t HOST_TOKEN_CHUNK = 16384;
+
+size_t elt_size(thanos_dtype_t d) { return d == THANOS_F32 ? 4 : 2; }
+bool dtype_ok(thanos_dtype_t d) { return d == THANOS_F32 || d == THANOS_BF16; }
+
+struct HostLayerLayout {
+  size_t H, U, xnorm, status, stats, Xstage, Win, Wout, mask, ws, ws_bytes, total;
+};
+
+HostLayerLayout host_layout(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
+  HostLayerLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off += round_up(bytes, 256);
+    return o;
+  };
+  L.H = take((size_t)b * b * 4);
+  L.U = take((size_t)b * b * 4);
+  L.xnorm = take((size_t)b * 4);
+  L.status = take(16);
+  L.stats = take(sizeof(thanos_stats_t));
+  L.Xstage = take(2 * (size_t)HOST_TOKEN_CHUNK * b * elt_size(dtype));
+  L.Win = take((size_t)c * b * elt_size(dtype));
+  L.Wout = take((size_t)c * b * elt_size(dtype));
+  L.mask = take((size_t)c * b);
+  size_t w = hessian_workspace_bytes(b, dtype);
+  size_t w2 = prepare_workspace_bytes(b);
+  size_t w3 = prune_workspace_bytes(c, b, B, dtype);
+  L.ws_bytes = w > w2 ? w : w2;
+  if (w3 > L.ws_bytes) L.ws_bytes = w3;
+  L.ws = take(L.ws_bytes);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+}  // namespace thanos
+
+using namespace thanos;
+
+extern "C" {
+
+thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
+                                          int64_t n_tok, int64_t ldx, void* workspace,
+                                          size_t ws_bytes, void* stream) {
+  if (!H || (!X && n_tok > 0)) return THANOS_ERR_INVALID_ARG;
+  if (!dtype_ok(xdtype)) return THANOS_ERR_DTYPE;
+  if (b < 8 || b > MAX_B || b % 8 != 0 || n_tok < 0) return THANOS_ERR_SHAPE;
+  if (ldx < b || ldx % 8 != 0) return THANOS_ERR_ALIGNMENT;
+  if (!aligned16(H) || !aligned16(X) || !aligned16(workspace)) return THANOS_ERR_ALIGNMENT;
+  if (n_tok == 0) return THANOS_OK;
+  if (ws_bytes < hessian_workspace_bytes(b, xdtype) || (!workspace && ws_bytes > 0))
+    return THANOS_ERR_WORKSPACE;
+  return hessian_accumulate_impl(H, b, X, xdtype, n_tok, ldx, workspace, ws_bytes,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prepare_inverse(const float* H, int64_t b, float damp_rel, float* factor,
+                                       float* xnorm, void* workspace, size_t ws_bytes,
+                                       int32_t* status_dev, void* stream) {
+  if (!H || !factor || !xnorm || !status_dev) return THANOS_ERR_INVALID_ARG;
+  if (!(damp_rel >= 0.f)) return THANOS_ERR_INVALID_ARG;
+  if (b < 8 || b > MAX_B || b % 8 != 0) return THANOS_ERR_SHAPE;
+  if (!aligned16(H) || !aligned16(factor) || !aligned16(xnorm) || !aligned16(workspace))
+    return THANOS_ERR_ALIGNMENT;
+  if (!workspace || ws_bytes < prepare_workspace_bytes(b)) return THANOS_ERR_WORKSPACE;
+  return prepare_inverse_impl(H, b, damp_rel, factor, xnorm, workspace, ws_bytes, status_dev,
+                              static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prune_layer(const void* W_in, void* W_out, uint8_t* mask_out,
+                                   thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                   const float* factor, const float* xnorm, thanos_mode_t mode,
+                                   double p, int32_t n, int32_t m, int32_t B, void* workspace,
+                                   size_t ws_bytes, thanos_stats_t* stats_dev, void* stream) {
+  if (!W_in || !W_out || !mask_out || !factor || !xnorm || !stats_dev)
+    return THANOS_ERR_INVALID_ARG;
+  if (!dtype_ok(wdtype)) return THANOS_ERR_DTYPE;
+  THANOS_TRY(validate_sweep_args(c, b, mode, p, n, m, B));
+  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(mask_out) || !aligned16(factor) ||
+      !aligned16(xnorm) || !aligned16(workspace) || !aligned16(stats_dev))
+    return THANOS_ERR_ALIGNMENT;
+  if (!workspace || ws_bytes < prune_workspace_bytes(c, b, B, wdtype)) return THANOS_ERR_WORKSPACE;
+  return prune_layer_impl(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, mode, p, n, m, B,
+                          workspace, ws_bytes, stats_dev, static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t b,
+                                   const float* factor, const float* xnorm, thanos_mode_t mode,
+                                   int32_t n, int32_t m, int32_t B, int64_t j1, int64_t* r_dev,
+                                   void* workspace, size_t ws_bytes, thanos_stats_t* stats_dev,
+                                   void* stream) {
+  if (!Wc || !mask || !factor || !xnorm || !stats_dev) return THANOS_ERR_INVALID_ARG;
+  if (mode == THANOS_UNSTRUCTURED && !r_dev) return THANOS_ERR_INVALID_ARG;
+  THANOS_TRY(validate_sweep_args(c, b, mode, 0.0, n, m, B));
+  if (j1 < 0 || j1 >= b || j1 % B != 0) return THANOS_ERR_SHAPE;
+  if (!aligned16(Wc) || !aligned16(mask) || !aligned16(factor) || !aligned16(xnorm) ||
+      !aligned16(workspace) || !aligned16(stats_dev))
+    return THANOS_ERR_ALIGNMENT;
+  if (!workspace || ws_bytes < prune_workspace_bytes(c, b, B, THANOS_F32))
+    return THANOS_ERR_WORKSPACE;
+  return prune_block_impl(Wc, mask, c, b, factor, xnorm, mode, n, m, B, j1, r_dev, workspace,
+                          ws_bytes, stats_dev, static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_host,
+                                        void* W_out_host, uint8_t* mask_out_host,
+                                        thanos_dtype_t dtype, int64_t c, int64_t b, int64_t a,
+                                        float damp_rel, thanos_mode_t mode, double p, int32_t n,
+                                        int32_t m, int32_t B, int32_t reuse_factor, void* arena,
+                                        size_t arena_bytes, thanos_stats_t* stats_host,
+                                        void* stream_v) {
+  if (!W_in_host || !W_out_host || !mask_out_host || !arena || !stats_host)
+    return THANOS_ERR_INVALID_ARG;
+  if (!reuse_factor && (!X_host || a < 1)) return THANOS_ERR_INVALID_ARG;
+  if (!dtype_ok(dtype)) return THANOS_ERR_DTYPE;
+  if (!(damp_rel >= 0.f)) return THANOS_ERR_INVALID_ARG;
+  if (b < 8 || b > MAX_B || b % 8 != 0) return THANOS_ERR_SHAPE;
+  THANOS_TRY(validate_sweep_args(c, b, mode, p, n, m, B));
+  if (!aligned16(arena)) return THANOS_ERR_ALIGNMENT;
+  HostLayerLayout L = host_layout(c, b, B, dtype);
+  if (arena_bytes < L.total) return THANOS_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  char* base = static_cast<char*>(arena);
+  float* H = reinterpret_cast<float*>(base + L.H);
+  float* U = reinterpret_cast<float*>(base + L.U);
+  float* xnorm = reinterpret_cast<float*>(base + L.xnorm);
+  int32_t* status = reinterpret_cast<int32_t*>(base + L.status);
+  thanos_stats_t* stats = reinterpret_cast<thanos_stats_t*>(base + L.stats);
+  void* ws = base + L.ws;
+  const size_t es = elt_size(dtype);
+
+  THANOS_CUDA(cudaMemcpyAsync(base + L.Win, W_in_host, (size_t)c * b * es, cudaMemcpyHostToDevice,
+                              stream));
+  if (!reuse_factor) {
+    THANOS_CUDA(cudaMemsetAsync(H, 0, (size_t)b * b * 4, stream));
+    THANOS_CUDA(cudaMemsetAsync(status, 0, 16, stream));
+    // Two staging buffers: the copy of chunk k+1 is issued on a second stream while chunk k is
+    // being accumulated.
+    cudaStream_t copy_stream;
+    cudaEvent_t copied[2], consumed[2];
+    THANOS_CUDA(cudaStreamCreateWithFlags(&copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming);
+      cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming);
+    }
+    cudaEvent_t start;
+    cudaEventCreateWithFlags(&start, cudaEventDisableTiming);
+    cudaEventRecord(start, stream);
+    cudaStreamWaitEvent(copy_stream, start, 0);
+    thanos_status_t st = THANOS_OK;
+    int64_t k = 0;
+    for (int64_t t0 = 0; t0 < a && st == THANOS_OK; t0 += HOST_TOKEN_CHUNK, ++k) {
+      int64_t nt = a - t0 < HOST_TOKEN_CHUNK ? a - t0 : HOST_TOKEN_CHUNK;
+      int slot = (int)(k & 1);
+      char* stage = base + L.Xstage + (size_t)slot * HOST_TOKEN_CHUNK * b * es;
+      if (k >= 2) cudaStreamWaitEvent(copy_stream, consumed[slot], 0);
+      if (cudaMemcpyAsync(stage, static_cast<const char*>(X_host) + (size_t)t0 * b * es,
+                          (size_t)nt * b * es, cudaMemcpyHostToDevice, copy_stream) != cudaSuccess)
+        st = THANOS_ERR_CUDA;
+      cudaEventRecord(copied[slot], copy_stream);
+      cudaStreamWaitEvent(stream, copied[slot], 0);
+      if (st == THANOS_OK)
+        st = thanos_hessian_accumulate(H, b, stage, dtype, nt, b, ws, L.ws_bytes, stream);
+      cudaEventRecord(consumed[slot], stream);
+    }
+    cudaStreamSynchronize(copy_stream);
+    cudaStreamDestroy(copy_stream);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(copied[i]);
+      cudaEventDestroy(consumed[i]);
+    }
+    cudaEventDestroy(start);
+    THANOS_TRY(st);
+    THANOS_TRY(thanos_prepare_inverse(H, b, damp_rel, U, xnorm, ws, L.ws_bytes, status, stream));
+  }
+  THANOS_TRY(thanos_prune_layer(base + L.Win, base + L.Wout, reinterpret_cast<uint8_t*>(base + L.mask),
+                                dtype, c, b, U, xnorm, mode, p, n, m, B, ws, L.ws_bytes, stats,
+                                stream));
+  THANOS_CUDA(cudaMemcpyAsync(W_out_host, base + L.Wout, (size_t)c * b * es, cudaMemcpyDeviceToHost,
+                              stream));
+  THANOS_CUDA(cudaMemcpyAsync(mask_out_host, base + L.mask, (size_t)c * b, cudaMemcpyDeviceToHost,
+                              stream));
+  THANOS_CUDA(cudaMemcpyAsync(stats_host, stats, sizeof(thanos_stats_t), cudaMemcpyDeviceToHost,
+                              stream));
+  int32_t st_host[4] = {0, 0, 0, 0};
+  THANOS_CUDA(cudaMemcpyAsync(st_host, status, 16, cudaMemcpyDeviceToHost, stream));
+  THANOS_CUDA(cudaStreamSynchronize(stream));
+  if (st_host[0] != 0 && stats_host->status == 0) {
+    stats_host->status = st_host[0];
+    stats_host->err_index = st_host[1];
+  }
+  return THANOS_OK;
+}
+
+size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
+  if (b < 8 || b > MAX_B || b % 8 != 0 || !dtype_ok(dtype)) return 0;
+  switch (which) {
+    case THANOS_WS_HESSIAN:
+      return hessian_workspace_bytes(b, dtype);
+    case THANOS_WS_PREPARE:
+      return prepare_workspace_bytes(b);
+    case THANOS_WS_PRUNE:
+      if (c < 1 || B < 1 || B > 512) return 0;
+      return prune_workspace_bytes(c, b, B, dtype);
+    case THANOS_WS_HOST_LAYER:
+      if (c < 1 || B < 1 || B > 512) return 0;
+      return host_layout(c, b, B, dtype).total;
+    default:
+      return 0;
+  }
+}
+
+const char* thanos_status_string(thanos_status_t status) {
+  switch (status) {
+    case THANOS_OK: return "ok";
+    case THANOS_ERR_INVALID_ARG: return "invalid argument";
+    case THANOS_ERR_SHAPE: return "unsupported shape";
+    case THANOS_ERR_DTYPE: return "unsupported dtype";
+    case THANOS_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+    case THANOS_ERR_WORKSPACE: return "workspace missing or too small";
+    case THANOS_ERR_NOT_SPD: return "matrix not positive definite";
+    case THANOS_ERR_TIMEOUT: return "device-side wait timed out";
+    case THANOS_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown status";
+  }
+}
+
+int32_t thanos_version(void) { return 100; }
+
+int64_t thanos_launch_count(void) { return (int64_t)g_launch_count.load(); }
+
+}  // extern "C"

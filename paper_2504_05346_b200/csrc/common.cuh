@@ -1,0 +1,70 @@
+// Shared host/device helpers of the Thanos sm_100a library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "thanos.h"
+
+namespace thanos {
+
+extern std::atomic<long long> g_launch_count;
+
+inline void count_launch(int n = 1) { g_launch_count.fetch_add(n, std::memory_order_relaxed); }
+
+// Launch check: cudaGetLastError right after a launch catches configuration errors only.
+#define THANOS_CHECK_LAUNCH()                               \
+  do {                                                      \
+    ::thanos::count_launch();                               \
+    if (cudaGetLastError() != cudaSuccess) return THANOS_ERR_CUDA; \
+  } while (0)
+
+#define THANOS_CUDA(call)                                   \
+  do {                                                      \
+    if ((call) != cudaSuccess) return THANOS_ERR_CUDA;      \
+  } while (0)
+
+#define THANOS_TRY(call)                                    \
+  do {                                                      \
+    thanos_status_t st__ = (call);                          \
+    if (st__ != THANOS_OK) return st__;                     \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Bump allocator over the caller's workspace (256-byte granules).
+struct Arena {
+  char* base;
+  size_t size;
+  size_t off;
+  Arena(void* p, size_t n) : base(static_cast<char*>(p)), size(n), off(0) {}
+  template <typename T>
+  T* take(size_t count) {
+    size_t bytes = round_up(count * sizeof(T), 256);
+    if (base == nullptr || off + bytes > size) {
+      off = size + 1;
+      return nullptr;
+    }
+    T* r = reinterpret_cast<T*>(base + off);
+    off += bytes;
+    return r;
+  }
+  bool ok() const { return off <= size; }
+};
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// First device-detected error wins.
+__device__ __forceinline__ void report_error(int32_t* status2, int32_t code, int32_t index) {
+  if (atomicCAS(status2, 0, code) == 0) status2[1] = index;
+}
+
+}  // namespace thanos

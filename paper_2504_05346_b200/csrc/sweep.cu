@@ -1,0 +1,658 @@
+// The block sweep of Algorithm 1 (unstructured) and Algorithm 4 (n:m, alpha = 0):
+// per block of B columns -- metric, mask, per-row solve, update of all columns to the right.
+//
+// With U from thanos_prepare_inverse, rows j1..j2 of inv(H_d[j1:, j1:]) are
+//   P = U_bb^T U[j1:j2, j1:]   (U_bb = U[j1:j2, j1:j2]),   G = P[:, 0:B] = U_bb^T U_bb,
+// so for a row with removed positions q (Eqs. 5-7): R = P[q, :], R-hat = G[q, q], u = w[q];
+// lambda-hat solves lambda-hat R-hat = u and the update is w - lambda-hat R (Eq. 8).  Writing
+// the multipliers of all rows as a c x B matrix Lambda (zero off the mask) turns the update of
+// the whole block into one dense product:  W[:, j1:] -= Lambda P.
+#include "simt_gemm.cuh"
+
+namespace thanos {
+
+namespace {
+
+constexpr int P0_BITS = 11, P1_BITS = 10, P2_BITS = 10;  // 31 key bits (metric >= 0)
+constexpr int HIST_BINS = 1 << P0_BITS;
+
+struct SweepState {
+  long long r;                   // removals still to place before the current block
+  unsigned long long k_rem;      // rank still to resolve inside the current candidate bin
+  unsigned long long need_eq;    // how many entries with key == tau are removed
+  unsigned long long count_eq;   // how many entries with key == tau the residual holds
+  unsigned long long blk_count;  // entries removed in the current block
+  unsigned int prefix;           // key bits fixed so far
+  unsigned int tau;              // threshold key of the current block
+  int none;                      // nothing to remove in this block
+  int pad;
+};
+
+__device__ __forceinline__ unsigned metric_key(float w, float xn) {
+  // |w| * ||X_j|| in fp32; non-negative floats order like their bit patterns
+  return __float_as_uint(fabsf(w) * xn);
+}
+
+// ------------------------------------------------------------------ P = U_bb^T U[j1:j2, j1:]
+__global__ void __launch_bounds__(256)
+pblock_kernel(const float* __restrict__ U, float* __restrict__ P, int b, int j1, int Bw) {
+  using G = SimtGemm<64, 64, 16, 4, 4, true, false, float, float>;
+  __shared__ float smem[G::SMEM_FLOATS];
+  const int N = b - j1;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  float acc[4][4] = {};
+  const float* Ub = U + (int64_t)j1 * b + j1;
+  // A(m, k) = U[j1 + k, j1 + m] vanishes for k > m
+  int kend = m0 + 64 < Bw ? m0 + 64 : Bw;
+  G::run(Ub, b, Ub, b, Bw, N, m0, n0, 0, kend, acc, smem);
+  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int gm = m0 + G::row_of(ty, i);
+    if (gm >= Bw) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int gn = n0 + G::col_of(tx, j);
+      if (gn < N) P[(int64_t)gm * b + j1 + gn] = acc[i][j];
+    }
+  }
+}
+
+// ------------------------------------------------------------------ unstructured selection
+__global__ void begin_block_kernel(SweepState* st, const int64_t* r_ext) {
+  if (r_ext) st->r = *r_ext;
+  st->none = (st->r <= 0) ? 1 : 0;
+  st->k_rem = st->r > 0 ? (unsigned long long)st->r : 0ull;
+  st->prefix = 0;
+  st->blk_count = 0;
+  st->need_eq = 0;
+  st->count_eq = 0;
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(256)
+hist_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
+                 int j1, const SweepState* __restrict__ st, unsigned* __restrict__ hist) {
+  constexpr int BITS = PASS == 0 ? P0_BITS : (PASS == 1 ? P1_BITS : P2_BITS);
+  constexpr int SHIFT = PASS == 0 ? (P1_BITS + P2_BITS) : (PASS == 1 ? P2_BITS : 0);
+  constexpr int NBIN = 1 << BITS;
+  __shared__ unsigned sh[NBIN];
+  if (st->none) return;
+  for (int i = threadIdx.x; i < NBIN; i += 256) sh[i] = 0;
+  __syncthreads();
+  const unsigned prefix = st->prefix;
+  const int w4 = (b - j1) >> 2;
+  for (int row = blockIdx.x; row < c; row += gridDim.x) {
+    const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+    const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
+    for (int q = threadIdx.x; q < w4; q += 256) {
+      float4 w = wr[q];
+      float4 x = __ldg(&xr[q]);
+      unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
+                       metric_key(w.w, x.w)};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (PASS == 0 || (k[e] >> (SHIFT + BITS)) == prefix)
+          atomicAdd(&sh[(k[e] >> SHIFT) & (NBIN - 1)], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < NBIN; i += 256)
+    if (sh[i]) atomicAdd(&hist[i], sh[i]);
+}
+
+// One CTA: locate the bin holding the k_rem-th smallest candidate, extend the prefix.
+template <int PASS>
+__global__ void __launch_bounds__(1024)
+scan_pass_kernel(SweepState* st, unsigned* __restrict__ hist) {
+  constexpr int BITS = PASS == 0 ? P0_BITS : (PASS == 1 ? P1_BITS : P2_BITS);
+  constexpr int NBIN = 1 << BITS;
+  constexpr int PER = (NBIN + 1023) / 1024;
+  __shared__ unsigned long long wsum[32];
+  if (st->none) return;
+  const int tid = threadIdx.x;
+  unsigned long long loc[PER];
+  unsigned long long tsum = 0;
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    int bin = tid * PER + e;
+    loc[e] = bin < NBIN ? hist[bin] : 0;
+    tsum += loc[e];
+  }
+  // inclusive scan of tsum over the block
+  unsigned long long inc = tsum;
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned long long v = __shfl_up_sync(0xffffffffu, inc, o);
+    if ((tid & 31) >= o) inc += v;
+  }
+  if ((tid & 31) == 31) wsum[tid >> 5] = inc;
+  __syncthreads();
+  if (tid < 32) {
+    unsigned long long v = wsum[tid];
+    unsigned long long s = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned long long u = __shfl_up_sync(0xffffffffu, s, o);
+      if (tid >= o) s += u;
+    }
+    wsum[tid] = s - v;  // exclusive prefix of warp totals
+  }
+  __syncthreads();
+  const unsigned long long k = st->k_rem;
+  unsigned long long excl = wsum[tid >> 5] + inc - tsum;
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    int bin = tid * PER + e;
+    if (bin < NBIN && excl < k && k <= excl + loc[e]) {
+      const unsigned np = (st->prefix << BITS) | (unsigned)bin;
+      st->prefix = np;
+      st->k_rem = k - excl;
+      if (PASS == 2) {
+        st->tau = np;
+        st->need_eq = k - excl;
+        st->count_eq = loc[e];
+      }
+    }
+    excl += loc[e];
+  }
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    int bin = tid * PER + e;
+    if (bin < NBIN) hist[bin] = 0;
+  }
+}
+
+// Rows' counts of entries equal to the threshold over the residual (only needed when the
+// tie-break has to leave some of them unpruned).
+__global__ void __launch_bounds__(256)
+tie_count_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
+                 int j1, const SweepState* __restrict__ st, unsigned* __restrict__ rowcnt) {
+  if (st->none || st->need_eq == st->count_eq) return;
+  __shared__ unsigned red[8];
+  const unsigned tau = st->tau;
+  const int w4 = (b - j1) >> 2;
+  for (int row = blockIdx.x; row < c; row += gridDim.x) {
+    const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+    const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
+    unsigned cnt = 0;
+    for (int q = threadIdx.x; q < w4; q += 256) {
+      float4 w = wr[q];
+      float4 x = __ldg(&xr[q]);
+      cnt += (metric_key(w.x, x.x) == tau) + (metric_key(w.y, x.y) == tau) +
+             (metric_key(w.z, x.z) == tau) + (metric_key(w.w, x.w) == tau);
+    }
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned t = 0;
+      for (int i = 0; i < 8; ++i) t += red[i];
+      rowcnt[row] = t;
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+tie_scan_kernel(int c, const SweepState* __restrict__ st, const unsigned* __restrict__ rowcnt,
+                unsigned long long* __restrict__ rowbase) {
+  if (st->none || st->need_eq == st->count_eq) return;
+  __shared__ unsigned long long wsum[32];
+  __shared__ unsigned long long carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < c; base += 1024) {
+    int row = base + threadIdx.x;
+    unsigned long long v = row < c ? rowcnt[row] : 0;
+    unsigned long long inc = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned long long u = __shfl_up_sync(0xffffffffu, inc, o);
+      if ((threadIdx.x & 31) >= o) inc += u;
+    }
+    if ((threadIdx.x & 31) == 31) wsum[threadIdx.x >> 5] = inc;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      unsigned long long t = wsum[threadIdx.x], s = t;
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long u = __shfl_up_sync(0xffffffffu, s, o);
+        if (threadIdx.x >= o) s += u;
+      }
+      wsum[threadIdx.x] = s - t;
+    }
+    __syncthreads();
+    unsigned long long excl = carry + wsum[threadIdx.x >> 5] + inc - v;
+    if (row < c) rowbase[row] = excl;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = excl + v;
+    __syncthreads();
+  }
+}
+
+// One warp per row: set the block's mask bytes.  key < tau -> removed; key == tau -> removed
+// while the (row, column)-ordered rank of the tie is below need_eq.
+__global__ void __launch_bounds__(256)
+mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
+                  uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, SweepState* st,
+                  const unsigned long long* __restrict__ rowbase, thanos_stats_t* stats) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const bool none = st->none != 0;
+  const unsigned tau = st->tau;
+  const bool all_ties = st->need_eq == st->count_eq;
+  const unsigned long long need = st->need_eq;
+  unsigned long long total = 0;
+  int smax = 0;
+  for (int row = blockIdx.x * 8 + warp; row < c; row += gridDim.x * 8) {
+    unsigned long long rank = (none || all_ties) ? 0ull : rowbase[row];
+    int s = 0;
+    for (int base = 0; base < Bw; base += 32) {
+      int jj = base + lane;
+      bool in = jj < Bw;
+      unsigned key = 0xffffffffu;
+      if (in) key = metric_key(Wc[(int64_t)row * b + j1 + jj], __ldg(&xnorm[j1 + jj]));
+      bool tie = in && !none && key == tau;
+      unsigned tb = __ballot_sync(0xffffffffu, tie);
+      bool pr = in && !none && key < tau;
+      if (tie) {
+        unsigned long long myrank = rank + __popc(tb & ((1u << lane) - 1u));
+        pr = all_ties || myrank < need;
+      }
+      rank += __popc(tb);
+      if (in) mask[(int64_t)row * b + j1 + jj] = pr ? 1 : 0;
+      s += __popc(__ballot_sync(0xffffffffu, pr));
+    }
+    total += s;
+    smax = s > smax ? s : smax;
+  }
+  if (lane == 0) {
+    if (total) atomicAdd(&st->blk_count, total);
+    if (smax) atomicMax(&stats->max_s, smax);
+  }
+}
+
+// n:m: one thread per (row, group of m columns); the n smallest keys, lower column on ties.
+__global__ void __launch_bounds__(256)
+nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
+               uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, int n, int m) {
+  const int groups = Bw / m;
+  int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= (int64_t)c * groups) return;
+  int row = (int)(idx / groups), g = (int)(idx % groups);
+  const float* w = Wc + (int64_t)row * b + j1 + g * m;
+  const float* x = xnorm + j1 + g * m;
+  unsigned key[32];
+  for (int e = 0; e < m; ++e) key[e] = metric_key(w[e], __ldg(&x[e]));
+  uint8_t* mo = mask + (int64_t)row * b + j1 + g * m;
+  for (int e = 0; e < m; ++e) {
+    // rank of e = number of entries that come before it in (key, column) order
+    int rk = 0;
+    for (int f = 0; f < m; ++f) rk += (key[f] < key[e]) || (key[f] == key[e] && f < e);
+    mo[e] = rk < n ? 1 : 0;
+  }
+}
+
+__global__ void finish_block_kernel(SweepState* st, thanos_stats_t* stats, int64_t* r_ext,
+                                    long long nm_count, int is_nm) {
+  unsigned long long cnt = is_nm ? (unsigned long long)nm_count : st->blk_count;
+  if (!is_nm) {
+    st->r -= (long long)cnt;
+    stats->r_left = st->r;
+    if (!st->none) {
+      stats->n_tied += (long long)(st->count_eq - st->need_eq);
+      stats->last_threshold_bits = st->tau;
+    }
+    if (r_ext) *r_ext = st->r;
+  }
+  stats->n_pruned += (long long)cnt;
+  stats->n_blocks += 1;
+  st->blk_count = 0;
+}
+
+// ------------------------------------------------------------------ per-row gather + solve
+// One warp per row.  Shared memory per warp: packed lower triangle of R-hat (s(s+1)/2 floats),
+// the right-hand side (s floats) and the index list q (s shorts).
+__global__ void __launch_bounds__(256)
+solve_rows_kernel(const float* __restrict__ Wc, const uint8_t* __restrict__ mask,
+                  const float* __restrict__ P, float* __restrict__ Lam, int c, int b, int j1,
+                  int Bw, int ldl, int smax, int is_nm, thanos_stats_t* stats) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int warps = blockDim.x >> 5;
+  const size_t tri = (size_t)smax * (smax + 1) / 2;
+  const size_t per_warp = ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
+  float* L = reinterpret_cast<float*>(dyn + per_warp * warp);
+  float* y = L + tri;
+  short* q = reinterpret_cast<short*>(y + smax);
+
+  for (int row = blockIdx.x * warps + warp; row < c; row += gridDim.x * warps) {
+    // q = phi(mask row): ascending positions of the removed entries inside the block
+    int s = 0;
+    for (int base = 0; base < Bw; base += 32) {
+      int jj = base + lane;
+      bool mb = jj < Bw && mask[(int64_t)row * b + j1 + jj] != 0;
+      unsigned bal = __ballot_sync(0xffffffffu, mb);
+      if (mb) {
+        int pos = s + __popc(bal & ((1u << lane) - 1u));
+        if (pos < smax) q[pos] = (short)jj;
+      }
+      s += __popc(bal);
+    }
+    for (int jj = lane; jj < Bw; jj += 32) Lam[(int64_t)row * ldl + jj] = 0.f;
+    if (s > smax) {  // cannot happen for a valid mask; refuse rather than overrun
+      if (lane == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
+      s = 0;
+    }
+    __syncwarp();
+    if (s == 0) continue;
+    if (is_nm && row == 0 && lane == 0) atomicMax(&stats->max_s, s);
+    // gather R-hat = G[q, q] (lower triangle) and u = w[q]
+    for (int a = 0; a < s; ++a) {
+      const float* Prow = P + (int64_t)q[a] * b + j1;
+      float* Lrow = L + (size_t)a * (a + 1) / 2;
+      for (int bb = lane; bb <= a; bb += 32) Lrow[bb] = Prow[q[bb]];
+    }
+    for (int a = lane; a < s; a += 32) y[a] = Wc[(int64_t)row * b + j1 + q[a]];
+    __syncwarp();
+    // Cholesky R-hat = L L^T, column by column
+    bool bad = false;
+    for (int j = 0; j < s; ++j) {
+      float* Lj = L + (size_t)j * (j + 1) / 2;
+      float part = 0.f;
+      for (int k = lane; k < j; k += 32) part = fmaf(Lj[k], Lj[k], part);
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      float d = Lj[j] - part;
+      if (!(d > 0.f) || !isfinite(d)) {
+        bad = true;
+        d = 1.f;
+      }
+      float ljj = sqrtf(d);
+      float inv = 1.f / ljj;
+      __syncwarp();
+      if (lane == 0) Lj[j] = ljj;
+      for (int i = j + 1 + lane; i < s; i += 32) {
+        float* Li = L + (size_t)i * (i + 1) / 2;
+        float v = Li[j];
+        for (int k = 0; k < j; ++k) v = fmaf(-Li[k], Lj[k], v);
+        Li[j] = v * inv;
+      }
+      __syncwarp();
+    }
+    if (bad) {
+      if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
+      continue;
+    }
+    // forward substitution L z = u (column oriented)
+    for (int j = 0; j < s; ++j) {
+      float zj = y[j] / L[(size_t)j * (j + 1) / 2 + j];
+      __syncwarp();
+      if (lane == 0) y[j] = zj;
+      for (int i = j + 1 + lane; i < s; i += 32)
+        y[i] = fmaf(-L[(size_t)i * (i + 1) / 2 + j], zj, y[i]);
+      __syncwarp();
+    }
+    // back substitution L^T lambda = z
+    for (int j = s - 1; j >= 0; --j) {
+      const float* Lj = L + (size_t)j * (j + 1) / 2;
+      float xj = y[j] / Lj[j];
+      __syncwarp();
+      if (lane == 0) y[j] = xj;
+      for (int k = lane; k < j; k += 32) y[k] = fmaf(-Lj[k], xj, y[k]);
+      __syncwarp();
+    }
+    for (int a = lane; a < s; a += 32) Lam[(int64_t)row * ldl + q[a]] = y[a];
+    __syncwarp();
+  }
+}
+
+// ------------------------------------------------------------------ W[:, j1:] -= Lambda P
+__global__ void __launch_bounds__(256)
+update_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
+              const float* __restrict__ Lam, const float* __restrict__ P, int c, int b, int j1,
+              int Bw, int ldl) {
+  using G = SimtGemm<128, 128, 16, 8, 8, false, false, float, float>;
+  __shared__ float smem[G::SMEM_FLOATS];
+  const int N = b - j1;
+  const int m0 = blockIdx.y * 128, n0 = blockIdx.x * 128;
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+  G::run(Lam, ldl, P + j1, b, c, N, m0, n0, 0, Bw, acc, smem);
+  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int gm = m0 + G::row_of(ty, i);
+    if (gm >= c) continue;
+#pragma unroll
+    for (int cj = 0; cj < 2; ++cj) {
+      int gn = n0 + G::col_of(tx, cj * 4);
+      if (gn >= N) continue;  // N and gn are multiples of 4
+      float4* wp = reinterpret_cast<float4*>(Wc + (int64_t)gm * b + j1 + gn);
+      float4 w = *wp;
+      w.x -= acc[i][cj * 4 + 0];
+      w.y -= acc[i][cj * 4 + 1];
+      w.z -= acc[i][cj * 4 + 2];
+      w.w -= acc[i][cj * 4 + 3];
+      if (gn < Bw) {
+        uchar4 mk = *reinterpret_cast<const uchar4*>(mask + (int64_t)gm * b + j1 + gn);
+        if (mk.x) w.x = 0.f;
+        if (mk.y) w.y = 0.f;
+        if (mk.z) w.z = 0.f;
+        if (mk.w) w.w = 0.f;
+      }
+      *wp = w;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ dtype conversion
+__global__ void to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out,
+                              int64_t n) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) out[i] = __bfloat162float(in[i]);
+}
+
+__global__ void to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out,
+                               int64_t n) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+__global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long long r) {
+  st->r = r;
+  st->k_rem = 0;
+  st->need_eq = st->count_eq = st->blk_count = 0;
+  st->prefix = st->tau = 0;
+  st->none = 0;
+  thanos_stats_t z = {};
+  z.r_left = r;
+  *stats = z;
+}
+
+struct SweepWs {
+  float* Wc;  // fp32 working copy when the I/O dtype is not fp32
+  float* P;
+  float* Lam;
+  unsigned* hist;
+  SweepState* st;
+  unsigned* rowcnt;
+  unsigned long long* rowbase;
+};
+
+size_t solve_per_warp_bytes(int smax) {
+  size_t tri = (size_t)smax * (smax + 1) / 2;
+  return ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
+}
+
+constexpr size_t SOLVE_SMEM_BUDGET = 220 * 1024;
+
+bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, int32_t B,
+           bool need_wc) {
+  Arena ar(workspace, ws_bytes);
+  w.Wc = need_wc ? ar.take<float>((size_t)c * b) : nullptr;
+  w.P = ar.take<float>((size_t)B * b);
+  w.Lam = ar.take<float>((size_t)c * B);
+  w.hist = ar.take<unsigned>(HIST_BINS);
+  w.st = ar.take<SweepState>(1);
+  w.rowcnt = ar.take<unsigned>((size_t)c);
+  w.rowbase = ar.take<unsigned long long>((size_t)c);
+  return ar.ok();
+}
+
+thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* U,
+                           const float* xnorm, thanos_mode_t mode, int n, int m, int B, int j1,
+                           int64_t* r_ext, const SweepWs& w, thanos_stats_t* stats,
+                           cudaStream_t stream) {
+  const int Bw = (b - j1 < B) ? b - j1 : B;
+  const int N = b - j1;
+  {
+    dim3 g((unsigned)ceil_div(N, 64), (unsigned)ceil_div(Bw, 64));
+    pblock_kernel<<<g, 256, 0, stream>>>(U, w.P, b, j1, Bw);
+    THANOS_CHECK_LAUNCH();
+  }
+  int smax;
+  if (mode == THANOS_UNSTRUCTURED) {
+    smax = Bw;
+    int hg = c < 148 * 8 ? c : 148 * 8;
+    begin_block_kernel<<<1, 1, 0, stream>>>(w.st, r_ext);
+    THANOS_CHECK_LAUNCH();
+    hist_pass_kernel<0><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    scan_pass_kernel<0><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    hist_pass_kernel<1><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    scan_pass_kernel<1><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    hist_pass_kernel<2><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    scan_pass_kernel<2><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
+    THANOS_CHECK_LAUNCH();
+    tie_scan_kernel<<<1, 1024, 0, stream>>>(c, w.st, w.rowcnt, w.rowbase);
+    THANOS_CHECK_LAUNCH();
+    int mg = (int)ceil_div(c, 8);
+    if (mg > 148 * 8) mg = 148 * 8;
+    mark_block_kernel<<<mg, 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
+                                              stats);
+    THANOS_CHECK_LAUNCH();
+  } else {
+    smax = Bw / m * n;
+    int64_t items = (int64_t)c * (Bw / m);
+    nm_mark_kernel<<<(unsigned)ceil_div(items, 256), 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1,
+                                                                      Bw, n, m);
+    THANOS_CHECK_LAUNCH();
+  }
+  {
+    if (smax < 1) smax = 1;
+    size_t per_warp = solve_per_warp_bytes(smax);
+    int warps = (int)(SOLVE_SMEM_BUDGET / per_warp);
+    if (warps < 1) return THANOS_ERR_SHAPE;
+    if (warps > 8) warps = 8;
+    size_t smem = per_warp * warps;
+    THANOS_CUDA(cudaFuncSetAttribute(solve_rows_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)SOLVE_SMEM_BUDGET));
+    int64_t grid = ceil_div(c, warps);
+    if (grid > 148 * 4) grid = 148 * 4;
+    solve_rows_kernel<<<(unsigned)grid, warps * 32, smem, stream>>>(
+        Wc, mask, w.P, w.Lam, c, b, j1, Bw, B, smax, mode == THANOS_NM ? 1 : 0, stats);
+    THANOS_CHECK_LAUNCH();
+  }
+  {
+    dim3 g((unsigned)ceil_div(N, 128), (unsigned)ceil_div(c, 128));
+    update_kernel<<<g, 256, 0, stream>>>(Wc, mask, w.Lam, w.P, c, b, j1, Bw, B);
+    THANOS_CHECK_LAUNCH();
+  }
+  long long nm_count = mode == THANOS_NM ? (long long)c * (Bw / m) * n : 0;
+  finish_block_kernel<<<1, 1, 0, stream>>>(w.st, stats, r_ext, nm_count, mode == THANOS_NM);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+}  // namespace
+
+size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
+  size_t t = 0;
+  if (dtype != THANOS_F32) t += round_up((size_t)c * b * sizeof(float), 256);
+  t += round_up((size_t)B * b * sizeof(float), 256);
+  t += round_up((size_t)c * B * sizeof(float), 256);
+  t += round_up(HIST_BINS * sizeof(unsigned), 256);
+  t += round_up(sizeof(SweepState), 256);
+  t += round_up((size_t)c * sizeof(unsigned), 256);
+  t += round_up((size_t)c * sizeof(unsigned long long), 256);
+  return t + 256;
+}
+
+thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, double p, int32_t n,
+                                    int32_t m, int32_t B) {
+  if (c < 1 || b < 1 || c > (1 << 30) || b > (1 << 30)) return THANOS_ERR_SHAPE;
+  if (b % 8 != 0 || B < 1 || B > 512 || B % 8 != 0) return THANOS_ERR_SHAPE;
+  if (mode == THANOS_UNSTRUCTURED) {
+    if (!(p >= 0.0 && p < 1.0)) return THANOS_ERR_INVALID_ARG;
+    if (solve_per_warp_bytes(B) > SOLVE_SMEM_BUDGET) return THANOS_ERR_SHAPE;
+  } else if (mode == THANOS_NM) {
+    if (!(n > 0 && n < m && m <= 32)) return THANOS_ERR_INVALID_ARG;
+    if (B % m != 0 || b % m != 0) return THANOS_ERR_SHAPE;
+    if (solve_per_warp_bytes(B / m * n) > SOLVE_SMEM_BUDGET) return THANOS_ERR_SHAPE;
+  } else {
+    return THANOS_ERR_INVALID_ARG;
+  }
+  return THANOS_OK;
+}
+
+thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b, const float* U,
+                                 const float* xnorm, thanos_mode_t mode, int32_t n, int32_t m,
+                                 int32_t B, int64_t j1, int64_t* r_dev, void* workspace,
+                                 size_t ws_bytes, thanos_stats_t* stats, cudaStream_t stream) {
+  SweepWs w;
+  if (!carve(w, workspace, ws_bytes, c, b, B, false)) return THANOS_ERR_WORKSPACE;
+  THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
+  THANOS_CUDA(cudaMemsetAsync(w.st, 0, sizeof(SweepState), stream));
+  return block_step(Wc, mask, (int)c, (int)b, U, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
+                    stream);
+}
+
+thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+                                 thanos_dtype_t wdtype, int64_t c, int64_t b, const float* U,
+                                 const float* xnorm, thanos_mode_t mode, double p, int32_t n,
+                                 int32_t m, int32_t B, void* workspace, size_t ws_bytes,
+                                 thanos_stats_t* stats, cudaStream_t stream) {
+  SweepWs w;
+  const bool need_wc = wdtype != THANOS_F32;
+  if (!carve(w, workspace, ws_bytes, c, b, B, need_wc)) return THANOS_ERR_WORKSPACE;
+  const int64_t nel = c * b;
+  float* Wc;
+  if (need_wc) {
+    Wc = w.Wc;
+    to_f32_kernel<<<148 * 8, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(W_in), Wc, nel);
+    THANOS_CHECK_LAUNCH();
+  } else {
+    Wc = static_cast<float*>(W_out);
+    if (W_in != W_out)
+      THANOS_CUDA(cudaMemcpyAsync(W_out, W_in, (size_t)nel * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, stream));
+  }
+  THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
+  long long r = 0;
+  if (mode == THANOS_UNSTRUCTURED) r = (long long)floor(p * (double)c * (double)b);
+  init_sweep_kernel<<<1, 1, 0, stream>>>(w.st, stats, r);
+  THANOS_CHECK_LAUNCH();
+  for (int64_t j1 = 0; j1 < b; j1 += B) {
+    THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, U, xnorm, mode, n, m, B, (int)j1, nullptr,
+                          w, stats, stream));
+  }
+  if (need_wc) {
+    to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(Wc, static_cast<__nv_bfloat16*>(W_out), nel);
+    THANOS_CHECK_LAUNCH();
+  }
+  return THANOS_OK;
+}
+
+}  // namespace thanos
