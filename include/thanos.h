@@ -77,11 +77,15 @@ typedef struct {
  * calibration chunks is the un-averaged d-sample Hessian of Appendix A.4).
  *
  *  H       device, fp32 [b, b], full symmetric storage; the caller zeroes it before the first
- *          chunk.  Updated in place; stays exactly symmetric.
+ *          chunk.  Updated in place.  H[i][j] and H[j][i] receive the same addends, but in an
+ *          unspecified order, so they may differ in the last bits; this library's own
+ *          consumers read the upper triangle only.
  *  X       device, [n_tok, b] tokens-major (the transpose of the paper's X), element type
  *          `xdtype`, leading dimension `ldx` elements (ldx >= b, ldx % 8 == 0).
  *  b % 8 == 0, n_tok >= 0 (0 is a no-op).
- *  workspace: thanos_workspace_bytes(THANOS_WS_HESSIAN, 0, b, 0, xdtype) bytes.
+ *  workspace: thanos_workspace_bytes(THANOS_WS_HESSIAN, 0, b, 0, xdtype) bytes.  Its first int32
+ *          is this call's device status word: cleared when the call starts, set to
+ *          THANOS_ERR_TIMEOUT if a bounded wait inside the tensor-core kernel ran out.
  * May be called any number of times; the order of floating-point summation across a call's
  * internal token slices is not fixed, so results can differ in the last bits between runs.
  */

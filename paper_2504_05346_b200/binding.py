@@ -271,3 +271,4 @@ def prune_layer_host(W_host: torch.Tensor, X_host: Optional[torch.Tensor], damp_
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_host (index %d)" % st.err_index)
     return out, mask, st
+

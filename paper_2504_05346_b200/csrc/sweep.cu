@@ -13,8 +13,11 @@ namespace thanos {
 
 namespace {
 
-constexpr int P0_BITS = 11, P1_BITS = 10, P2_BITS = 10;  // 31 key bits (metric >= 0)
-constexpr int HIST_BINS = 1 << P0_BITS;
+// Radix select over the 31 significant key bits (metric >= 0): four passes of 8, 8, 8, 7 bits.
+constexpr int NPASS = 4;
+constexpr int HIST_BINS = 256;
+__host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
+__host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0)); }
 
 struct SweepState {
   long long r;                   // removals still to place before the current block
@@ -69,22 +72,25 @@ __global__ void begin_block_kernel(SweepState* st, const int64_t* r_ext) {
   st->count_eq = 0;
 }
 
+// Histogram of one radix digit over the residual.  The shared histogram keeps one counter per
+// (bin, lane): a warp never hits the same bank twice, whatever the skew of the metric.
 template <int PASS>
 __global__ void __launch_bounds__(256)
 hist_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                  int j1, const SweepState* __restrict__ st, unsigned* __restrict__ hist) {
-  constexpr int BITS = PASS == 0 ? P0_BITS : (PASS == 1 ? P1_BITS : P2_BITS);
-  constexpr int SHIFT = PASS == 0 ? (P1_BITS + P2_BITS) : (PASS == 1 ? P2_BITS : 0);
+  constexpr int BITS = pass_bits(PASS);
+  constexpr int SHIFT = pass_shift(PASS);
   constexpr int NBIN = 1 << BITS;
-  __shared__ unsigned sh[NBIN];
+  __shared__ unsigned sh[NBIN * 32];
   if (st->none) return;
-  for (int i = threadIdx.x; i < NBIN; i += 256) sh[i] = 0;
+  for (int i = threadIdx.x; i < NBIN * 32; i += 256) sh[i] = 0;
   __syncthreads();
   const unsigned prefix = st->prefix;
+  const int lane = threadIdx.x & 31;
   const int w4 = (b - j1) >> 2;
+  const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
   for (int row = blockIdx.x; row < c; row += gridDim.x) {
     const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-    const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
     for (int q = threadIdx.x; q < w4; q += 256) {
       float4 w = wr[q];
       float4 x = __ldg(&xr[q]);
@@ -93,62 +99,53 @@ hist_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, 
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         if (PASS == 0 || (k[e] >> (SHIFT + BITS)) == prefix)
-          atomicAdd(&sh[(k[e] >> SHIFT) & (NBIN - 1)], 1u);
+          atomicAdd(&sh[((k[e] >> SHIFT) & (NBIN - 1)) * 32 + lane], 1u);
       }
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < NBIN; i += 256)
-    if (sh[i]) atomicAdd(&hist[i], sh[i]);
+  for (int bin = threadIdx.x; bin < NBIN; bin += 256) {
+    unsigned t = 0;
+#pragma unroll
+    for (int l = 0; l < 32; ++l) t += sh[bin * 32 + ((l + bin) & 31)];
+    if (t) atomicAdd(&hist[bin], t);
+  }
 }
 
-// One CTA: locate the bin holding the k_rem-th smallest candidate, extend the prefix.
+// One warp: locate the bin holding the k_rem-th smallest candidate, extend the prefix.
 template <int PASS>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(32)
 scan_pass_kernel(SweepState* st, unsigned* __restrict__ hist) {
-  constexpr int BITS = PASS == 0 ? P0_BITS : (PASS == 1 ? P1_BITS : P2_BITS);
+  constexpr int BITS = pass_bits(PASS);
   constexpr int NBIN = 1 << BITS;
-  constexpr int PER = (NBIN + 1023) / 1024;
-  __shared__ unsigned long long wsum[32];
+  constexpr int PER = HIST_BINS / 32;
   if (st->none) return;
-  const int tid = threadIdx.x;
+  const int lane = threadIdx.x;
   unsigned long long loc[PER];
   unsigned long long tsum = 0;
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
-    int bin = tid * PER + e;
+    int bin = lane * PER + e;
     loc[e] = bin < NBIN ? hist[bin] : 0;
     tsum += loc[e];
   }
-  // inclusive scan of tsum over the block
   unsigned long long inc = tsum;
   for (int o = 1; o < 32; o <<= 1) {
     unsigned long long v = __shfl_up_sync(0xffffffffu, inc, o);
-    if ((tid & 31) >= o) inc += v;
+    if (lane >= o) inc += v;
   }
-  if ((tid & 31) == 31) wsum[tid >> 5] = inc;
-  __syncthreads();
-  if (tid < 32) {
-    unsigned long long v = wsum[tid];
-    unsigned long long s = v;
-    for (int o = 1; o < 32; o <<= 1) {
-      unsigned long long u = __shfl_up_sync(0xffffffffu, s, o);
-      if (tid >= o) s += u;
-    }
-    wsum[tid] = s - v;  // exclusive prefix of warp totals
-  }
-  __syncthreads();
   const unsigned long long k = st->k_rem;
-  unsigned long long excl = wsum[tid >> 5] + inc - tsum;
-  __syncthreads();
+  const unsigned prefix = st->prefix;
+  __syncwarp();
+  unsigned long long excl = inc - tsum;
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
-    int bin = tid * PER + e;
+    int bin = lane * PER + e;
     if (bin < NBIN && excl < k && k <= excl + loc[e]) {
-      const unsigned np = (st->prefix << BITS) | (unsigned)bin;
+      const unsigned np = (prefix << BITS) | (unsigned)bin;
       st->prefix = np;
       st->k_rem = k - excl;
-      if (PASS == 2) {
+      if (PASS == NPASS - 1) {
         st->tau = np;
         st->need_eq = k - excl;
         st->count_eq = loc[e];
@@ -157,10 +154,7 @@ scan_pass_kernel(SweepState* st, unsigned* __restrict__ hist) {
     excl += loc[e];
   }
 #pragma unroll
-  for (int e = 0; e < PER; ++e) {
-    int bin = tid * PER + e;
-    if (bin < NBIN) hist[bin] = 0;
-  }
+  for (int e = 0; e < PER; ++e) hist[lane * PER + e] = 0;
 }
 
 // Rows' counts of entries equal to the threshold over the residual (only needed when the
@@ -523,15 +517,19 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     THANOS_CHECK_LAUNCH();
     hist_pass_kernel<0><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
     THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<0><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    scan_pass_kernel<0><<<1, 32, 0, stream>>>(w.st, w.hist);
     THANOS_CHECK_LAUNCH();
     hist_pass_kernel<1><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
     THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<1><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    scan_pass_kernel<1><<<1, 32, 0, stream>>>(w.st, w.hist);
     THANOS_CHECK_LAUNCH();
     hist_pass_kernel<2><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
     THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<2><<<1, 1024, 0, stream>>>(w.st, w.hist);
+    scan_pass_kernel<2><<<1, 32, 0, stream>>>(w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    hist_pass_kernel<3><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
+    THANOS_CHECK_LAUNCH();
+    scan_pass_kernel<3><<<1, 32, 0, stream>>>(w.st, w.hist);
     THANOS_CHECK_LAUNCH();
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
     THANOS_CHECK_LAUNCH();
