@@ -178,6 +178,38 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
                                         size_t arena_bytes, thanos_stats_t* stats_host,
                                         void* stream);
 
+/*
+ * Variant of thanos_prune_layer for callers that cannot provide a workspace.  The paper has no
+ * counterpart of this call; it computes exactly what thanos_prune_layer computes.
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -- a plugin
+ * inside a serving process whose allocator already owns the whole GPU, a step of a pipeline
+ * that must not call cudaMalloc because that call synchronises the device and would stall
+ * the other streams, or a host that forbids allocation after start-up.  Such a caller has its
+ * weights, the factor and the outputs, but no spare buffer to pass as `workspace`.
+ *
+ * The sweep's scratch is a fixed 4 MiB array that is part of the library's device image
+ * (every GPU that loads the library holds it until the process exits).  The call allocates
+ * nothing and frees nothing.  A layer fits when
+ *     thanos_workspace_bytes(THANOS_WS_PRUNE, c, b, B, wdtype) <= 4 MiB
+ * (for example 512 x 512 fp32 with B = 128, or 256 x 1024 bf16 with B = 64); anything larger
+ * is refused with THANOS_ERR_WORKSPACE before any work is enqueued.
+ *
+ * The first call on a device looks up the device address of that array (once per device, with
+ * the device current); make this first call before starting any stream capture.  All calls
+ * on a device share the one array: the call clears the parts that must start from zero, so
+ * leftovers of an earlier call are harmless, but two calls that overlap on the GPU (different
+ * streams, or different host threads) race on it -- serialise them.
+ *
+ * Arguments, layouts, results and device-side error reporting are those of
+ * thanos_prune_layer, minus `workspace` and `ws_bytes`.
+ */
+thanos_status_t thanos_prune_layer_noalloc(const void* W_in, void* W_out, uint8_t* mask_out,
+                                           thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                           const float* factor, const float* xnorm,
+                                           thanos_mode_t mode, double p, int32_t n, int32_t m,
+                                           int32_t B, thanos_stats_t* stats_dev, void* stream);
+
 /* Minimum workspace in bytes for a call (see thanos_ws_which_t); 0 for unsupported shapes. */
 size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
 

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     prune_layer,
     prune_block,
     prune_layer_host,
+    prune_layer_noalloc,
     workspace_bytes,
     launch_count,
     status_string,

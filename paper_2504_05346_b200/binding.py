@@ -90,6 +90,9 @@ def load_library():
                                             i32, ctypes.c_double, i32, i32, i32, i32, vp, sz,
                                             ctypes.POINTER(_Stats), vp]
     lib.thanos_prune_layer_host.restype = i32
+    lib.thanos_prune_layer_noalloc.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, i32,
+                                               ctypes.c_double, i32, i32, i32, vp, vp]
+    lib.thanos_prune_layer_noalloc.restype = i32
     lib.thanos_workspace_bytes.argtypes = [i32, i64, i64, i32, i32]
     lib.thanos_workspace_bytes.restype = sz
     lib.thanos_status_string.argtypes = [i32]
@@ -272,3 +275,27 @@ def prune_layer_host(W_host: torch.Tensor, X_host: Optional[torch.Tensor], damp_
         raise ThanosError(st.status, "thanos_prune_layer_host (index %d)" % st.err_index)
     return out, mask, st
 
+
+def prune_layer_noalloc(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tensor, mode: int,
+                        p: float = 0.0, n: int = 0, m: int = 0, B: int = 128, stream=None,
+                        out: Optional[torch.Tensor] = None, mask: Optional[torch.Tensor] = None):
+    """thanos_prune_layer_noalloc: the sweep with the library's built-in 4 MiB scratch, for
+    callers that cannot allocate a workspace.  Only the outputs are created here (pass `out`
+    and `mask` to avoid even that).  Calls on one device must not overlap."""
+    lib = load_library()
+    _check_dev(W, factor, xnorm)
+    c, b = W.shape
+    dt = _dtype_code(W)
+    if out is None:
+        out = torch.empty_like(W)
+    if mask is None:
+        mask = torch.empty((c, b), dtype=torch.uint8, device=W.device)
+    stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
+    _check(lib.thanos_prune_layer_noalloc(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
+                                          factor.data_ptr(), xnorm.data_ptr(), mode, float(p), n,
+                                          m, B, stats.data_ptr(), _stream_ptr(stream)),
+           "thanos_prune_layer_noalloc")
+    st = _read_stats(stats)
+    if st.status != 0:
+        raise ThanosError(st.status, "thanos_prune_layer_noalloc (row %d)" % st.err_index)
+    return out, mask, st

@@ -1,0 +1,68 @@
+"""thanos_prune_layer_noalloc -- the sweep for callers that cannot allocate a workspace (their
+allocator owns the whole GPU, or a cudaMalloc would stall their other streams).  It must give
+what thanos_prune_layer gives, call after call, although every call reuses the same built-in
+scratch array.  Collected last on purpose: a run that stops at the first failure has then
+already run every other test."""
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def T():
+    import paper_2504_05346_b200 as T_
+    from paper_2504_05346_b200 import build as B_
+
+    B_.build()
+    T_.load_library()
+    return T_
+
+
+def _factor(T, b, seed):
+    Xt = WL.make_activations(2048, b, "f32", "student_t4", 0.02, 0, 10.0, seed, 0, mix=0.5).to(DEV)
+    H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(H, Xt)
+    return T.prepare_inverse(H, 0.01)
+
+
+def test_noalloc_matches_prune_layer_on_consecutive_calls(T):
+    # call 1: fp32 weights, unstructured; call 2 right after it: bf16 weights (which also keeps
+    # its fp32 working copy in the shared scratch), 2:4 -- different shapes, same scratch array
+    U1, xn1 = _factor(T, 256, seed=3)
+    W1 = WL.make_weight(64, 256, "f32", seed=71).to(DEV)
+    U2, xn2 = _factor(T, 128, seed=4)
+    W2 = WL.make_weight(48, 128, "bf16", seed=72).to(DEV)
+
+    a1 = T.prune_layer_noalloc(W1, U1, xn1, T.UNSTRUCTURED, p=0.5, B=64)
+    a2 = T.prune_layer_noalloc(W2, U2, xn2, T.NM, n=2, m=4, B=32)
+    a3 = T.prune_layer_noalloc(W1, U1, xn1, T.UNSTRUCTURED, p=0.5, B=64)  # and back again
+    torch.cuda.synchronize()
+    r1 = T.prune_layer(W1, U1, xn1, T.UNSTRUCTURED, p=0.5, B=64)
+    r2 = T.prune_layer(W2, U2, xn2, T.NM, n=2, m=4, B=32)
+
+    for got, ref in ((a1, r1), (a2, r2), (a3, r1)):
+        assert torch.equal(got[1], ref[1])  # masks bit for bit
+        g, r = got[0].double().cpu().numpy(), ref[0].double().cpu().numpy()
+        assert np.linalg.norm(g - r) <= 1e-6 * np.linalg.norm(r)
+        assert got[2].n_pruned == ref[2].n_pruned and got[2].status == 0
+    assert a1[2].n_pruned == 64 * 256 // 2 and a2[2].n_pruned == 48 * 128 // 2
+
+
+def test_noalloc_refuses_layers_beyond_its_fixed_scratch(T):
+    U, xn = _factor(T, 256, seed=5)
+    big = torch.zeros((8192, 256), dtype=torch.float32, device=DEV)  # needs > 4 MiB of scratch
+    assert T.workspace_bytes(2, 8192, 256, 128, T.F32) > 4 << 20
+    with pytest.raises(T.ThanosError) as e:
+        T.prune_layer_noalloc(big, U, xn, T.UNSTRUCTURED, p=0.5, B=128)
+    assert e.value.code == 5  # THANOS_ERR_WORKSPACE, nothing was launched
+    # a layer that fits still works afterwards
+    W = WL.make_weight(32, 256, "f32", seed=73).to(DEV)
+    out, mask, st = T.prune_layer_noalloc(W, U, xn, T.NM, n=2, m=4, B=64)
+    assert st.n_pruned == 32 * 256 // 2
