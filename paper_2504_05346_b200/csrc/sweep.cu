@@ -1,15 +1,26 @@
 // The block sweep of Algorithm 1 (unstructured) and Algorithm 4 (n:m, alpha = 0):
 // per block of B columns -- metric, mask, per-row solve, update of all columns to the right.
 //
-// With U from thanos_prepare_inverse, rows j1..j2 of inv(H_d[j1:, j1:]) are
-//   P = U_bb^T U[j1:j2, j1:]   (U_bb = U[j1:j2, j1:j2]),   G = P[:, 0:B] = U_bb^T U_bb,
-// so for a row with removed positions q (Eqs. 5-7): R = P[q, :], R-hat = G[q, q], u = w[q];
-// lambda-hat solves lambda-hat R-hat = u and the update is w - lambda-hat R (Eq. 8).  Writing
-// the multipliers of all rows as a c x B matrix Lambda (zero off the mask) turns the update of
-// the whole block into one dense product:  W[:, j1:] -= Lambda P.
+// With U from thanos_prepare_inverse (U^T U = inv(H_d), upper) the residual inverse of a block
+// starting at j1 is U[j1:, j1:]^T U[j1:, j1:].  Per block, with U_bb = U[j1:j2, j1:j2] and
+// V_bb = inv(U_bb):
+//   G = U_bb^T U_bb      the block of the residual inverse (R-hat = G[q, q] in Eqs. 5-7),
+//   S = V_bb V_bb^T      its inverse, for rows that remove more than half of the block,
+//   P2 = V_bb U[j1:j2, j2:]
+// and Eq. 8 splits into the change of the block itself, delta (c x B, from the per-row solves;
+// delta_q = -w_q), and the change of every column to the right, which is the dense product
+//   W[:, j2:] += delta P2      (because -lambda-hat R = delta inv(G) (U_bb^T U[j1:j2, j1:])).
+// G, S, V_bb and P2 depend only on U, so they are computed for all blocks at the start of the
+// sweep.
 #include "simt_gemm.cuh"
 
 namespace thanos {
+
+bool solve_supported(int s_direct_max, int n_small_max);
+thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                   int ld_mat, float* D, int c, int b, int j1, int Bw, int ldd,
+                                   int s_fixed, const int* row_lists, const unsigned* list_counts,
+                                   thanos_stats_t* stats, cudaStream_t stream);
 
 namespace {
 
@@ -36,33 +47,99 @@ __device__ __forceinline__ unsigned metric_key(float w, float xn) {
   return __float_as_uint(fabsf(w) * xn);
 }
 
-// ------------------------------------------------------------------ P = U_bb^T U[j1:j2, j1:]
+// ------------------------------------------------------------------ per-block matrices
+// One CTA per block: dense copy of U_bb (zeros below the diagonal) and V_bb = inv(U_bb) by back
+// substitution, one column of V_bb per thread, accumulated in double.
+__global__ void __launch_bounds__(512)
+block_inverse_kernel(const float* __restrict__ U, float* __restrict__ Ubb, float* __restrict__ Vbb,
+                     int b, int B) {
+  const int bb = blockIdx.x;
+  const int j1 = bb * B;
+  const int Bw = (b - j1 < B) ? b - j1 : B;
+  float* Uo = Ubb + (size_t)bb * B * B;
+  float* Vo = Vbb + (size_t)bb * B * B;
+  for (int e = threadIdx.x; e < B * B; e += blockDim.x) {
+    const int i = e / B, j = e - i * B;
+    float u = 0.f;
+    if (i < Bw && j < Bw && j >= i) u = U[(int64_t)(j1 + i) * b + j1 + j];
+    Uo[e] = u;
+    Vo[e] = 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < Bw; j += blockDim.x) {
+    // column j of V: U_bb v = e_j, from row j upwards
+    Vo[(size_t)j * B + j] = 1.f / Uo[(size_t)j * B + j];
+    for (int i = j - 1; i >= 0; --i) {
+      double acc = 0.0;
+      for (int k = i + 1; k <= j; ++k)
+        acc += (double)Uo[(size_t)i * B + k] * (double)Vo[(size_t)k * B + j];
+      Vo[(size_t)i * B + j] = (float)(-acc / (double)Uo[(size_t)i * B + i]);
+    }
+  }
+}
+
+// which = 0: G = U_bb^T U_bb;  which = 1: S = V_bb V_bb^T.  Grid (B/64, B/64, blocks).
+template <int WHICH>
 __global__ void __launch_bounds__(256)
-pblock_kernel(const float* __restrict__ U, float* __restrict__ P, int b, int j1, int Bw) {
-  using G = SimtGemm<64, 64, 16, 4, 4, true, false, float, float>;
+block_gram_kernel(const float* __restrict__ Fbb, float* __restrict__ Out, int b, int B) {
+  using G = SimtGemm<64, 64, 16, 4, 4, WHICH == 0, WHICH == 1, float, float>;
   __shared__ float smem[G::SMEM_FLOATS];
-  const int N = b - j1;
+  const int bb = blockIdx.z;
+  const int j1 = bb * B;
+  const int Bw = (b - j1 < B) ? b - j1 : B;
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  if (m0 >= Bw || n0 >= Bw) return;
+  const float* F = Fbb + (size_t)bb * B * B;
   float acc[4][4] = {};
-  const float* Ub = U + (int64_t)j1 * b + j1;
-  // A(m, k) = U[j1 + k, j1 + m] vanishes for k > m
-  int kend = m0 + 64 < Bw ? m0 + 64 : Bw;
-  G::run(Ub, b, Ub, b, Bw, N, m0, n0, 0, kend, acc, smem);
+  G::run(F, B, F, B, Bw, Bw, m0, n0, 0, Bw, acc, smem);
+  float* O = Out + (size_t)bb * B * B;
   const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    int gm = m0 + G::row_of(ty, i);
+    const int gm = m0 + G::row_of(ty, i);
     if (gm >= Bw) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      int gn = n0 + G::col_of(tx, j);
-      if (gn < N) P[(int64_t)gm * b + j1 + gn] = acc[i][j];
+      const int gn = n0 + G::col_of(tx, j);
+      if (gn < Bw) O[(size_t)gm * B + gn] = acc[i][j];
+    }
+  }
+}
+
+// P2[j1 + m, j2 + n] = sum_k V_bb[m, k] U[j1 + k, j2 + n] for every block.  Grid (n tiles of the
+// widest block, B/64, blocks).
+__global__ void __launch_bounds__(256)
+block_rows_kernel(const float* __restrict__ U, const float* __restrict__ Vbb,
+                  float* __restrict__ P2, int b, int B) {
+  using G = SimtGemm<64, 64, 16, 4, 4, false, false, float, float>;
+  __shared__ float smem[G::SMEM_FLOATS];
+  const int bb = blockIdx.z;
+  const int j1 = bb * B;
+  const int Bw = (b - j1 < B) ? b - j1 : B;
+  const int j2 = j1 + Bw;
+  const int N = b - j2;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  if (m0 >= Bw || n0 >= N) return;
+  float acc[4][4] = {};
+  // V_bb is upper-triangular: column k contributes to rows m <= k
+  G::run(Vbb + (size_t)bb * B * B, B, U + (int64_t)j1 * b + j2, b, Bw, N, m0, n0, m0, Bw, acc,
+         smem);
+  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gm = m0 + G::row_of(ty, i);
+    if (gm >= Bw) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gn = n0 + G::col_of(tx, j);
+      if (gn < N) P2[(int64_t)(j1 + gm) * b + j2 + gn] = acc[i][j];
     }
   }
 }
 
 // ------------------------------------------------------------------ unstructured selection
-__global__ void begin_block_kernel(SweepState* st, const int64_t* r_ext) {
+__global__ void begin_block_kernel(SweepState* st, const int64_t* r_ext, unsigned* list_counts) {
+  list_counts[0] = list_counts[1] = 0;
   if (r_ext) st->r = *r_ext;
   st->none = (st->r <= 0) ? 1 : 0;
   st->k_rem = st->r > 0 ? (unsigned long long)st->r : 0ull;
@@ -228,7 +305,8 @@ tie_scan_kernel(int c, const SweepState* __restrict__ st, const unsigned* __rest
 __global__ void __launch_bounds__(256)
 mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
                   uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, SweepState* st,
-                  const unsigned long long* __restrict__ rowbase, thanos_stats_t* stats) {
+                  const unsigned long long* __restrict__ rowbase, int* __restrict__ row_lists,
+                  unsigned* __restrict__ list_counts, thanos_stats_t* stats) {
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const bool none = st->none != 0;
@@ -258,6 +336,12 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
     }
     total += s;
     smax = s > smax ? s : smax;
+    if (lane == 0) {
+      // rows that remove more than half of the block are solved in the complement form
+      const int kind = (s > Bw - s) ? 1 : 0;
+      const unsigned pos = atomicAdd(&list_counts[kind], 1u);
+      row_lists[(size_t)kind * c + pos] = row;
+    }
   }
   if (lane == 0) {
     if (total) atomicAdd(&st->blk_count, total);
@@ -303,118 +387,21 @@ __global__ void finish_block_kernel(SweepState* st, thanos_stats_t* stats, int64
   st->blk_count = 0;
 }
 
-// ------------------------------------------------------------------ per-row gather + solve
-// One warp per row.  Shared memory per warp: packed lower triangle of R-hat (s(s+1)/2 floats),
-// the right-hand side (s floats) and the index list q (s shorts).
+// ------------------------------------------------------------------ W[:, j2:] += delta P2
 __global__ void __launch_bounds__(256)
-solve_rows_kernel(const float* __restrict__ Wc, const uint8_t* __restrict__ mask,
-                  const float* __restrict__ P, float* __restrict__ Lam, int c, int b, int j1,
-                  int Bw, int ldl, int smax, int is_nm, thanos_stats_t* stats) {
-  extern __shared__ __align__(16) unsigned char dyn[];
-  const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-  const int warps = blockDim.x >> 5;
-  const size_t tri = (size_t)smax * (smax + 1) / 2;
-  const size_t per_warp = ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
-  float* L = reinterpret_cast<float*>(dyn + per_warp * warp);
-  float* y = L + tri;
-  short* q = reinterpret_cast<short*>(y + smax);
-
-  for (int row = blockIdx.x * warps + warp; row < c; row += gridDim.x * warps) {
-    // q = phi(mask row): ascending positions of the removed entries inside the block
-    int s = 0;
-    for (int base = 0; base < Bw; base += 32) {
-      int jj = base + lane;
-      bool mb = jj < Bw && mask[(int64_t)row * b + j1 + jj] != 0;
-      unsigned bal = __ballot_sync(0xffffffffu, mb);
-      if (mb) {
-        int pos = s + __popc(bal & ((1u << lane) - 1u));
-        if (pos < smax) q[pos] = (short)jj;
-      }
-      s += __popc(bal);
-    }
-    for (int jj = lane; jj < Bw; jj += 32) Lam[(int64_t)row * ldl + jj] = 0.f;
-    if (s > smax) {  // cannot happen for a valid mask; refuse rather than overrun
-      if (lane == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
-      s = 0;
-    }
-    __syncwarp();
-    if (s == 0) continue;
-    if (is_nm && row == 0 && lane == 0) atomicMax(&stats->max_s, s);
-    // gather R-hat = G[q, q] (lower triangle) and u = w[q]
-    for (int a = 0; a < s; ++a) {
-      const float* Prow = P + (int64_t)q[a] * b + j1;
-      float* Lrow = L + (size_t)a * (a + 1) / 2;
-      for (int bb = lane; bb <= a; bb += 32) Lrow[bb] = Prow[q[bb]];
-    }
-    for (int a = lane; a < s; a += 32) y[a] = Wc[(int64_t)row * b + j1 + q[a]];
-    __syncwarp();
-    // Cholesky R-hat = L L^T, column by column
-    bool bad = false;
-    for (int j = 0; j < s; ++j) {
-      float* Lj = L + (size_t)j * (j + 1) / 2;
-      float part = 0.f;
-      for (int k = lane; k < j; k += 32) part = fmaf(Lj[k], Lj[k], part);
-      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-      float d = Lj[j] - part;
-      if (!(d > 0.f) || !isfinite(d)) {
-        bad = true;
-        d = 1.f;
-      }
-      float ljj = sqrtf(d);
-      float inv = 1.f / ljj;
-      __syncwarp();
-      if (lane == 0) Lj[j] = ljj;
-      for (int i = j + 1 + lane; i < s; i += 32) {
-        float* Li = L + (size_t)i * (i + 1) / 2;
-        float v = Li[j];
-        for (int k = 0; k < j; ++k) v = fmaf(-Li[k], Lj[k], v);
-        Li[j] = v * inv;
-      }
-      __syncwarp();
-    }
-    if (bad) {
-      if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
-      continue;
-    }
-    // forward substitution L z = u (column oriented)
-    for (int j = 0; j < s; ++j) {
-      float zj = y[j] / L[(size_t)j * (j + 1) / 2 + j];
-      __syncwarp();
-      if (lane == 0) y[j] = zj;
-      for (int i = j + 1 + lane; i < s; i += 32)
-        y[i] = fmaf(-L[(size_t)i * (i + 1) / 2 + j], zj, y[i]);
-      __syncwarp();
-    }
-    // back substitution L^T lambda = z
-    for (int j = s - 1; j >= 0; --j) {
-      const float* Lj = L + (size_t)j * (j + 1) / 2;
-      float xj = y[j] / Lj[j];
-      __syncwarp();
-      if (lane == 0) y[j] = xj;
-      for (int k = lane; k < j; k += 32) y[k] = fmaf(-Lj[k], xj, y[k]);
-      __syncwarp();
-    }
-    for (int a = lane; a < s; a += 32) Lam[(int64_t)row * ldl + q[a]] = y[a];
-    __syncwarp();
-  }
-}
-
-// ------------------------------------------------------------------ W[:, j1:] -= Lambda P
-__global__ void __launch_bounds__(256)
-update_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
-              const float* __restrict__ Lam, const float* __restrict__ P, int c, int b, int j1,
-              int Bw, int ldl) {
+update_kernel(float* __restrict__ Wc, const float* __restrict__ D, const float* __restrict__ P2,
+              int c, int b, int j1, int Bw, int ldd) {
   using G = SimtGemm<128, 128, 16, 8, 8, false, false, float, float>;
   __shared__ float smem[G::SMEM_FLOATS];
-  const int N = b - j1;
+  const int j2 = j1 + Bw;
+  const int N = b - j2;
   const int m0 = blockIdx.y * 128, n0 = blockIdx.x * 128;
   float acc[8][8];
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-  G::run(Lam, ldl, P + j1, b, c, N, m0, n0, 0, Bw, acc, smem);
+  G::run(D, ldd, P2 + (int64_t)j1 * b + j2, b, c, N, m0, n0, 0, Bw, acc, smem);
   const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -424,19 +411,12 @@ update_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     for (int cj = 0; cj < 2; ++cj) {
       int gn = n0 + G::col_of(tx, cj * 4);
       if (gn >= N) continue;  // N and gn are multiples of 4
-      float4* wp = reinterpret_cast<float4*>(Wc + (int64_t)gm * b + j1 + gn);
+      float4* wp = reinterpret_cast<float4*>(Wc + (int64_t)gm * b + j2 + gn);
       float4 w = *wp;
-      w.x -= acc[i][cj * 4 + 0];
-      w.y -= acc[i][cj * 4 + 1];
-      w.z -= acc[i][cj * 4 + 2];
-      w.w -= acc[i][cj * 4 + 3];
-      if (gn < Bw) {
-        uchar4 mk = *reinterpret_cast<const uchar4*>(mask + (int64_t)gm * b + j1 + gn);
-        if (mk.x) w.x = 0.f;
-        if (mk.y) w.y = 0.f;
-        if (mk.z) w.z = 0.f;
-        if (mk.w) w.w = 0.f;
-      }
+      w.x += acc[i][cj * 4 + 0];
+      w.y += acc[i][cj * 4 + 1];
+      w.z += acc[i][cj * 4 + 2];
+      w.w += acc[i][cj * 4 + 3];
       *wp = w;
     }
   }
@@ -469,51 +449,70 @@ __global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long lo
 }
 
 struct SweepWs {
-  float* Wc;  // fp32 working copy when the I/O dtype is not fp32
-  float* P;
-  float* Lam;
+  float* Wc;   // fp32 working copy when the I/O dtype is not fp32
+  float* D;    // [c, B] change of the current block (delta)
+  float* Ubb;  // [blocks, B, B] per-block matrices
+  float* Vbb;
+  float* G;
+  float* S;
+  float* P2;   // [b, b]; rows of block j1..j2 hold V_bb U[j1:j2, j2:] in columns >= j2
   unsigned* hist;
   SweepState* st;
   unsigned* rowcnt;
   unsigned long long* rowbase;
+  int* row_lists;         // [2, c] rows of the current block by kind of system
+  unsigned* list_counts;  // [2]
 };
-
-size_t solve_per_warp_bytes(int smax) {
-  size_t tri = (size_t)smax * (smax + 1) / 2;
-  return ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
-}
-
-constexpr size_t SOLVE_SMEM_BUDGET = 220 * 1024;
 
 bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, int32_t B,
            bool need_wc) {
   Arena ar(workspace, ws_bytes);
+  const size_t blocks = (size_t)ceil_div(b, B);
   w.Wc = need_wc ? ar.take<float>((size_t)c * b) : nullptr;
-  w.P = ar.take<float>((size_t)B * b);
-  w.Lam = ar.take<float>((size_t)c * B);
+  w.D = ar.take<float>((size_t)c * B);
+  w.Ubb = ar.take<float>(blocks * B * B);
+  w.Vbb = ar.take<float>(blocks * B * B);
+  w.G = ar.take<float>(blocks * B * B);
+  w.S = ar.take<float>(blocks * B * B);
+  w.P2 = ar.take<float>((size_t)b * b);
   w.hist = ar.take<unsigned>(HIST_BINS);
   w.st = ar.take<SweepState>(1);
   w.rowcnt = ar.take<unsigned>((size_t)c);
   w.rowbase = ar.take<unsigned long long>((size_t)c);
+  w.row_lists = ar.take<int>(2 * (size_t)c);
+  w.list_counts = ar.take<unsigned>(2);
   return ar.ok();
 }
 
-thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* U,
-                           const float* xnorm, thanos_mode_t mode, int n, int m, int B, int j1,
-                           int64_t* r_ext, const SweepWs& w, thanos_stats_t* stats,
-                           cudaStream_t stream) {
-  const int Bw = (b - j1 < B) ? b - j1 : B;
-  const int N = b - j1;
-  {
-    dim3 g((unsigned)ceil_div(N, 64), (unsigned)ceil_div(Bw, 64));
-    pblock_kernel<<<g, 256, 0, stream>>>(U, w.P, b, j1, Bw);
+// G, S, V_bb of every block and P2, once per sweep.
+thanos_status_t prepare_blocks(const float* U, int b, int B, const SweepWs& w,
+                               cudaStream_t stream) {
+  const int blocks = (int)ceil_div(b, B);
+  block_inverse_kernel<<<blocks, B < 128 ? 128 : B, 0, stream>>>(U, w.Ubb, w.Vbb, b, B);
+  THANOS_CHECK_LAUNCH();
+  dim3 gg((unsigned)ceil_div(B, 64), (unsigned)ceil_div(B, 64), (unsigned)blocks);
+  block_gram_kernel<0><<<gg, 256, 0, stream>>>(w.Ubb, w.G, b, B);
+  THANOS_CHECK_LAUNCH();
+  block_gram_kernel<1><<<gg, 256, 0, stream>>>(w.Vbb, w.S, b, B);
+  THANOS_CHECK_LAUNCH();
+  if (b > B) {
+    dim3 gp((unsigned)ceil_div(b - B, 64), (unsigned)ceil_div(B, 64), (unsigned)blocks);
+    block_rows_kernel<<<gp, 256, 0, stream>>>(U, w.Vbb, w.P2, b, B);
     THANOS_CHECK_LAUNCH();
   }
-  int smax;
+  return THANOS_OK;
+}
+
+thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* xnorm,
+                           thanos_mode_t mode, int n, int m, int B, int j1, int64_t* r_ext,
+                           const SweepWs& w, thanos_stats_t* stats, cudaStream_t stream) {
+  const int Bw = (b - j1 < B) ? b - j1 : B;
+  const int j2 = j1 + Bw;
+  const int bb = j1 / B;
+  int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    smax = Bw;
     int hg = c < 148 * 8 ? c : 148 * 8;
-    begin_block_kernel<<<1, 1, 0, stream>>>(w.st, r_ext);
+    begin_block_kernel<<<1, 1, 0, stream>>>(w.st, r_ext, w.list_counts);
     THANOS_CHECK_LAUNCH();
     hist_pass_kernel<0><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
     THANOS_CHECK_LAUNCH();
@@ -538,34 +537,21 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     int mg = (int)ceil_div(c, 8);
     if (mg > 148 * 8) mg = 148 * 8;
     mark_block_kernel<<<mg, 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
-                                              stats);
+                                              w.row_lists, w.list_counts, stats);
     THANOS_CHECK_LAUNCH();
   } else {
-    smax = Bw / m * n;
+    s_fixed = Bw / m * n;
     int64_t items = (int64_t)c * (Bw / m);
     nm_mark_kernel<<<(unsigned)ceil_div(items, 256), 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1,
                                                                       Bw, n, m);
     THANOS_CHECK_LAUNCH();
   }
-  {
-    if (smax < 1) smax = 1;
-    size_t per_warp = solve_per_warp_bytes(smax);
-    int warps = (int)(SOLVE_SMEM_BUDGET / per_warp);
-    if (warps < 1) return THANOS_ERR_SHAPE;
-    if (warps > 8) warps = 8;
-    size_t smem = per_warp * warps;
-    THANOS_CUDA(cudaFuncSetAttribute(solve_rows_kernel,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)SOLVE_SMEM_BUDGET));
-    int64_t grid = ceil_div(c, warps);
-    if (grid > 148 * 4) grid = 148 * 4;
-    solve_rows_kernel<<<(unsigned)grid, warps * 32, smem, stream>>>(
-        Wc, mask, w.P, w.Lam, c, b, j1, Bw, B, smax, mode == THANOS_NM ? 1 : 0, stats);
-    THANOS_CHECK_LAUNCH();
-  }
-  {
-    dim3 g((unsigned)ceil_div(N, 128), (unsigned)ceil_div(c, 128));
-    update_kernel<<<g, 256, 0, stream>>>(Wc, mask, w.Lam, w.P, c, b, j1, Bw, B);
+  THANOS_TRY(launch_block_solve(Wc, mask, w.G + (size_t)bb * B * B, w.S + (size_t)bb * B * B, B,
+                                w.D, c, b, j1, Bw, B, s_fixed, w.row_lists, w.list_counts, stats,
+                                stream));
+  if (j2 < b) {
+    dim3 g((unsigned)ceil_div(b - j2, 128), (unsigned)ceil_div(c, 128));
+    update_kernel<<<g, 256, 0, stream>>>(Wc, w.D, w.P2, c, b, j1, Bw, B);
     THANOS_CHECK_LAUNCH();
   }
   long long nm_count = mode == THANOS_NM ? (long long)c * (Bw / m) * n : 0;
@@ -578,13 +564,17 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
 
 size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
   size_t t = 0;
+  const size_t blocks = (size_t)ceil_div(b, B);
   if (dtype != THANOS_F32) t += round_up((size_t)c * b * sizeof(float), 256);
-  t += round_up((size_t)B * b * sizeof(float), 256);
   t += round_up((size_t)c * B * sizeof(float), 256);
+  t += 4 * round_up(blocks * B * B * sizeof(float), 256);
+  t += round_up((size_t)b * b * sizeof(float), 256);
   t += round_up(HIST_BINS * sizeof(unsigned), 256);
   t += round_up(sizeof(SweepState), 256);
   t += round_up((size_t)c * sizeof(unsigned), 256);
   t += round_up((size_t)c * sizeof(unsigned long long), 256);
+  t += round_up(2 * (size_t)c * sizeof(int), 256);
+  t += 256;
   return t + 256;
 }
 
@@ -594,11 +584,12 @@ thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, do
   if (b % 8 != 0 || B < 1 || B > 512 || B % 8 != 0) return THANOS_ERR_SHAPE;
   if (mode == THANOS_UNSTRUCTURED) {
     if (!(p >= 0.0 && p < 1.0)) return THANOS_ERR_INVALID_ARG;
-    if (solve_per_warp_bytes(B) > SOLVE_SMEM_BUDGET) return THANOS_ERR_SHAPE;
+    if (!solve_supported(B, B / 2)) return THANOS_ERR_SHAPE;
   } else if (mode == THANOS_NM) {
     if (!(n > 0 && n < m && m <= 32)) return THANOS_ERR_INVALID_ARG;
     if (B % m != 0 || b % m != 0) return THANOS_ERR_SHAPE;
-    if (solve_per_warp_bytes(B / m * n) > SOLVE_SMEM_BUDGET) return THANOS_ERR_SHAPE;
+    const int s = B / m * n;
+    if (!solve_supported(s, s < B - s ? s : B - s)) return THANOS_ERR_SHAPE;
   } else {
     return THANOS_ERR_INVALID_ARG;
   }
@@ -613,7 +604,8 @@ thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b,
   if (!carve(w, workspace, ws_bytes, c, b, B, false)) return THANOS_ERR_WORKSPACE;
   THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
   THANOS_CUDA(cudaMemsetAsync(w.st, 0, sizeof(SweepState), stream));
-  return block_step(Wc, mask, (int)c, (int)b, U, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
+  THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
+  return block_step(Wc, mask, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
                     stream);
 }
 
@@ -642,9 +634,10 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
   if (mode == THANOS_UNSTRUCTURED) r = (long long)floor(p * (double)c * (double)b);
   init_sweep_kernel<<<1, 1, 0, stream>>>(w.st, stats, r);
   THANOS_CHECK_LAUNCH();
+  THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
   for (int64_t j1 = 0; j1 < b; j1 += B) {
-    THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, U, xnorm, mode, n, m, B, (int)j1, nullptr,
-                          w, stats, stream));
+    THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr, w,
+                          stats, stream));
   }
   if (need_wc) {
     to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(Wc, static_cast<__nv_bfloat16*>(W_out), nel);
