@@ -210,6 +210,28 @@ thanos_status_t thanos_prune_layer_noalloc(const void* W_in, void* W_out, uint8_
                                            thanos_mode_t mode, double p, int32_t n, int32_t m,
                                            int32_t B, thanos_stats_t* stats_dev, void* stream);
 
+/*
+ * Dense product on the tensor cores with fp32 accuracy:
+ *     D = (accumulate ? D : 0) + alpha * A * op(B)
+ * This is the contraction behind Eq. 8 applied to every row of a block at once (the change of the
+ * columns right of a block is delta times a matrix that depends only on the Hessian), exposed
+ * so that it can be checked and timed on its own.  Every fp32 operand is split into three bf16
+ * planes and six plane products are accumulated in fp32, so the result agrees with an fp32
+ * product to a few units of 2^-24 of sum |a||b|.
+ *
+ *  D   device fp32 [M, N], leading dimension ldd (ldd % 4 == 0).
+ *  A   device fp32 [M, K], leading dimension lda.
+ *  B   device fp32; b_transposed != 0: [N, K] (op(B) = B^T), else [K, N]; leading dimension ldb.
+ *  lda, ldb multiples of 4; K and the contiguous extent of B multiples of 4.
+ *  workspace: thanos_dense_product_workspace(M, N, K) bytes; its first int32 is the device status
+ *  word of the call (THANOS_ERR_TIMEOUT if a bounded wait ran out).
+ */
+thanos_status_t thanos_dense_product(float* D, int64_t ldd, const float* A, int64_t lda,
+                                     const float* B, int64_t ldb, int32_t b_transposed, int64_t M,
+                                     int64_t N, int64_t K, float alpha, int32_t accumulate,
+                                     void* workspace, size_t ws_bytes, void* stream);
+size_t thanos_dense_product_workspace(int64_t M, int64_t N, int64_t K);
+
 /* Minimum workspace in bytes for a call (see thanos_ws_which_t); 0 for unsupported shapes. */
 size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
 

@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     prune_block,
     prune_layer_host,
     prune_layer_noalloc,
+    dense_product,
     workspace_bytes,
     launch_count,
     status_string,

@@ -93,6 +93,11 @@ def load_library():
     lib.thanos_prune_layer_noalloc.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, i32,
                                                ctypes.c_double, i32, i32, i32, vp, vp]
     lib.thanos_prune_layer_noalloc.restype = i32
+    lib.thanos_dense_product.argtypes = [vp, i64, vp, i64, vp, i64, i32, i64, i64, i64,
+                                         ctypes.c_float, i32, vp, sz, vp]
+    lib.thanos_dense_product.restype = i32
+    lib.thanos_dense_product_workspace.argtypes = [i64, i64, i64]
+    lib.thanos_dense_product_workspace.restype = sz
     lib.thanos_workspace_bytes.argtypes = [i32, i64, i64, i32, i32]
     lib.thanos_workspace_bytes.restype = sz
     lib.thanos_status_string.argtypes = [i32]
@@ -299,3 +304,32 @@ def prune_layer_noalloc(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tens
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_noalloc (row %d)" % st.err_index)
     return out, mask, st
+
+
+def dense_product(A: torch.Tensor, B: torch.Tensor, b_transposed: bool = False, alpha: float = 1.0,
+                  out: Optional[torch.Tensor] = None, accumulate: bool = False, stream=None,
+                  check: bool = True):
+    """thanos_dense_product: out = (accumulate ? out : 0) + alpha * A @ (B^T if b_transposed
+    else B), fp32 device matrices (rows may be strided: the last dimension is contiguous)."""
+    lib = load_library()
+    _check_dev(A, B)
+    assert A.dtype == torch.float32 and B.dtype == torch.float32
+    assert A.stride(1) == 1 and B.stride(1) == 1
+    M, K = A.shape
+    N = B.shape[0] if b_transposed else B.shape[1]
+    assert (B.shape[1] if b_transposed else B.shape[0]) == K
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+        assert not accumulate
+    assert out.stride(1) == 1
+    nbytes = lib.thanos_dense_product_workspace(M, N, K)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=A.device)
+    _check(lib.thanos_dense_product(out.data_ptr(), out.stride(0), A.data_ptr(), A.stride(0),
+                                    B.data_ptr(), B.stride(0), 1 if b_transposed else 0, M, N, K,
+                                    float(alpha), 1 if accumulate else 0, ws.data_ptr(), nbytes,
+                                    _stream_ptr(stream)), "thanos_dense_product")
+    if check:
+        st = int(ws[:4].view(torch.int32).item())
+        if st != 0:
+            raise ThanosError(st, "thanos_dense_product (device)")
+    return out

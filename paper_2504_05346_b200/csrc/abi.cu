@@ -1,5 +1,6 @@
 // extern "C" entry points: argument checks, workspace carving, dispatch.
 #include "common.cuh"
+#include "tc_gemm.cuh"
 
 namespace thanos {
 
@@ -225,6 +226,61 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
     stats_host->err_index = st_host[1];
   }
   return THANOS_OK;
+}
+
+size_t thanos_dense_product_workspace(int64_t M, int64_t N, int64_t K) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  const size_t Kp = round_up((size_t)K, 8), Np = round_up((size_t)N, 8);
+  const size_t a = round_up(3 * (size_t)M * Kp * 2, 256);
+  const size_t bt = 3 * (size_t)N * Kp * 2, bn = 3 * (size_t)K * Np * 2;
+  return 256 + a + round_up(bt > bn ? bt : bn, 256);
+}
+
+thanos_status_t thanos_dense_product(float* D, int64_t ldd, const float* A, int64_t lda,
+                                     const float* B, int64_t ldb, int32_t b_transposed, int64_t M,
+                                     int64_t N, int64_t K, float alpha, int32_t accumulate,
+                                     void* workspace, size_t ws_bytes, void* stream_v) {
+  if (!D || !A || !B || !workspace) return THANOS_ERR_INVALID_ARG;
+  if (M < 1 || N < 1 || K < 1 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30))
+    return THANOS_ERR_SHAPE;
+  if (ldd % 4 || lda % 4 || ldb % 4 || K % 4 || (!b_transposed && N % 4)) return THANOS_ERR_ALIGNMENT;
+  if (ldd < N || lda < K || ldb < (b_transposed ? K : N)) return THANOS_ERR_SHAPE;
+  if (!aligned16(D) || !aligned16(A) || !aligned16(B) || !aligned16(workspace))
+    return THANOS_ERR_ALIGNMENT;
+  if (ws_bytes < thanos_dense_product_workspace(M, N, K)) return THANOS_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  const int64_t Kp = (int64_t)round_up((size_t)K, 8), Np = (int64_t)round_up((size_t)N, 8);
+  char* base = static_cast<char*>(workspace);
+  int32_t* status = reinterpret_cast<int32_t*>(base);
+  __nv_bfloat16* Ap = reinterpret_cast<__nv_bfloat16*>(base + 256);
+  __nv_bfloat16* Bp =
+      reinterpret_cast<__nv_bfloat16*>(base + 256 + round_up(3 * (size_t)M * Kp * 2, 256));
+  THANOS_CUDA(cudaMemsetAsync(status, 0, 16, stream));
+  THANOS_TRY(split3_planes(A, lda, M, K, Ap, Kp, M * Kp, stream));
+  TcGemmArgs g;
+  if (b_transposed) {
+    THANOS_TRY(split3_planes(B, ldb, N, K, Bp, Kp, N * Kp, stream));
+    g.ldb = Kp;
+    g.b_plane = N * Kp;
+  } else {
+    THANOS_TRY(split3_planes(B, ldb, K, N, Bp, Np, K * Np, stream));
+    g.ldb = Np;
+    g.b_plane = K * Np;
+  }
+  g.D = D;
+  g.ldd = ldd;
+  g.A = Ap;
+  g.lda = Kp;
+  g.a_plane = M * Kp;
+  g.B = Bp;
+  g.b_kmajor = b_transposed ? 1 : 0;
+  g.M = (int)M;
+  g.N = (int)N;
+  g.K = (int)K;
+  g.alpha = alpha;
+  g.accumulate = accumulate ? 1 : 0;
+  g.status = status;
+  return tc_gemm_split3(g, stream);
 }
 
 size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {

@@ -25,6 +25,16 @@ namespace {
 
 constexpr unsigned FULL = 0xffffffffu;
 
+// delta -> three bf16 planes (h, m, l) for the tensor-core update
+__device__ __forceinline__ void store_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
+#pragma unroll
+  for (int pl = 0; pl < 3; ++pl) {
+    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
+    p[(int64_t)pl * plane] = hb;
+    d -= __bfloat162float(hb);
+  }
+}
+
 __host__ __device__ __forceinline__ int tri_row_off(int r) {
   // rows 8m .. 8m+7 have 8m + 12 floats each (8m + 8 columns plus a 4-float skew)
   const int m = r >> 3, t = r & 7;
@@ -63,7 +73,8 @@ template <int NR>
 __global__ void __launch_bounds__(384)
 solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                        const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
-                       float* __restrict__ D, int c, int b, int j1, int Bw, int ldd, int panels,
+                       __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw, int ldd,
+                       int panels,
                        int mat_in_smem, const int* __restrict__ row_lists,
                        const unsigned* __restrict__ list_counts, int fixed_kind, int report_max_s,
                        thanos_stats_t* stats) {
@@ -175,7 +186,7 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         }
       }
       if (s == 0) {  // nothing removed: the row is not touched in this block
-        for (int jj = lane; jj < Bw; jj += 32) D[(int64_t)row * ldd + jj] = 0.f;
+        for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
         __syncwarp();
         continue;
       }
@@ -316,7 +327,7 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       }
       if (bad) {
         if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
-        for (int jj = lane; jj < Bw; jj += 32) D[(int64_t)row * ldd + jj] = 0.f;
+        for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
         __syncwarp();
         continue;
       }
@@ -402,7 +413,7 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         const float d = dvec[jj];
         const bool removed = mrow[jj] != 0;
         wrow[jj] = removed ? 0.f : wblk[jj] + d;
-        D[(int64_t)row * ldd + jj] = d;
+        store_split3(D + (int64_t)row * ldd + jj, dplane, d);
       }
       __syncwarp();
     }
@@ -413,8 +424,9 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
 // triangle in shared memory, column-by-column Cholesky, direct form only.
 __global__ void __launch_bounds__(256)
 solve_rows_general_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
-                          const float* __restrict__ G, int ldg, float* __restrict__ D, int c, int b,
-                          int j1, int Bw, int ldd, int smax, int report_max_s,
+                          const float* __restrict__ G, int ldg, __nv_bfloat16* __restrict__ D,
+                          int64_t dplane, int c, int b, int j1, int Bw, int ldd, int smax,
+                          int report_max_s,
                           thanos_stats_t* stats) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int lane = threadIdx.x & 31;
@@ -446,7 +458,7 @@ solve_rows_general_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ ma
     }
     __syncwarp();
     if (s == 0) {
-      for (int jj = lane; jj < Bw; jj += 32) D[(int64_t)row * ldd + jj] = 0.f;
+      for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
     if (report_max_s && row == 0 && lane == 0) atomicMax(&stats->max_s, s);
@@ -482,7 +494,7 @@ solve_rows_general_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ ma
     }
     if (bad) {
       if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
-      for (int jj = lane; jj < Bw; jj += 32) D[(int64_t)row * ldd + jj] = 0.f;
+      for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
     for (int j = 0; j < s; ++j) {
@@ -514,7 +526,7 @@ solve_rows_general_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ ma
         d = -g;
         wrow[jj] = w + d;
       }
-      D[(int64_t)row * ldd + jj] = d;
+      store_split3(D + (int64_t)row * ldd + jj, dplane, d);
     }
     __syncwarp();
   }
@@ -529,7 +541,8 @@ size_t general_per_warp_bytes(int smax) {
 
 template <int NR>
 thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, const float* S,
-                            int ld_mat, float* D, int c, int b, int j1, int Bw, int ldd, int n_max,
+                            int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1, int Bw,
+                            int ldd, int n_max,
                             const int* row_lists, const unsigned* list_counts, int fixed_kind,
                             int report_max_s, thanos_stats_t* stats, cudaStream_t stream) {
   const int panels = (n_max + 1 + 7) / 8;
@@ -545,7 +558,7 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
   int64_t grid = ceil_div(c, warps);
   if (grid > 148) grid = 148;
   solve_rows_fast_kernel<NR><<<(unsigned)grid, warps * 32, smem, stream>>>(
-      Wc, mask, G, S, ld_mat, D, c, b, j1, Bw, ldd, panels, in_smem ? 1 : 0, row_lists,
+      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, panels, in_smem ? 1 : 0, row_lists,
       list_counts, fixed_kind, report_max_s, stats);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
@@ -560,12 +573,13 @@ bool solve_supported(int s_direct_max, int n_small_max) {
 }
 
 // Solves every row of the block [j1, j1 + Bw): writes the block's new weights into Wc and the
-// change D (c x Bw, leading dimension ldd).  G and S are the block's Bw x Bw matrices (leading
+// change D (c x Bw as three bf16 planes dplane elements apart, leading dimension ldd).  G and S are the block's Bw x Bw matrices (leading
 // dimension ld_mat).  s_fixed >= 0 says every row removes exactly s_fixed entries (n:m);
 // otherwise row_lists[2][c] / list_counts[2] hold the rows sorted by kind (0: |q| <= |k|).
 thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
-                                   int ld_mat, float* D, int c, int b, int j1, int Bw, int ldd,
-                                   int s_fixed, const int* row_lists, const unsigned* list_counts,
+                                   int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
+                                   int Bw, int ldd, int s_fixed, const int* row_lists,
+                                   const unsigned* list_counts,
                                    thanos_stats_t* stats, cudaStream_t stream) {
   const bool uniform = s_fixed >= 0;
   const int n_small = uniform ? (s_fixed < Bw - s_fixed ? s_fixed : Bw - s_fixed) : Bw / 2;
@@ -581,7 +595,8 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
     int64_t grid = ceil_div(c, warps);
     if (grid > 148 * 4) grid = 148 * 4;
     solve_rows_general_kernel<<<(unsigned)grid, warps * 32, per_warp * warps, stream>>>(
-        Wc, mask, G, ld_mat, D, c, b, j1, Bw, ldd, smax < 1 ? 1 : smax, uniform ? 1 : 0, stats);
+        Wc, mask, G, ld_mat, D, dplane, c, b, j1, Bw, ldd, smax < 1 ? 1 : smax, uniform ? 1 : 0,
+        stats);
     THANOS_CHECK_LAUNCH();
     return THANOS_OK;
   }
@@ -590,12 +605,12 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
   const unsigned* lc = uniform ? nullptr : list_counts;
   const int rep = uniform ? 1 : 0;
   if (n_small + 1 <= 32)
-    return launch_fast<1>(Wc, mask, G, S, ld_mat, D, c, b, j1, Bw, ldd, n_small, rl, lc,
+    return launch_fast<1>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                           fixed_kind, rep, stats, stream);
   if (n_small + 1 <= 64)
-    return launch_fast<2>(Wc, mask, G, S, ld_mat, D, c, b, j1, Bw, ldd, n_small, rl, lc,
+    return launch_fast<2>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                           fixed_kind, rep, stats, stream);
-  return launch_fast<3>(Wc, mask, G, S, ld_mat, D, c, b, j1, Bw, ldd, n_small, rl, lc, fixed_kind,
+  return launch_fast<3>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc, fixed_kind,
                         rep, stats, stream);
 }
 

@@ -13,13 +13,15 @@
 // G, S, V_bb and P2 depend only on U, so they are computed for all blocks at the start of the
 // sweep.
 #include "simt_gemm.cuh"
+#include "tc_gemm.cuh"
 
 namespace thanos {
 
 bool solve_supported(int s_direct_max, int n_small_max);
 thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
-                                   int ld_mat, float* D, int c, int b, int j1, int Bw, int ldd,
-                                   int s_fixed, const int* row_lists, const unsigned* list_counts,
+                                   int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
+                                   int Bw, int ldd, int s_fixed, const int* row_lists,
+                                   const unsigned* list_counts,
                                    thanos_stats_t* stats, cudaStream_t stream);
 
 namespace {
@@ -110,7 +112,7 @@ block_gram_kernel(const float* __restrict__ Fbb, float* __restrict__ Out, int b,
 // widest block, B/64, blocks).
 __global__ void __launch_bounds__(256)
 block_rows_kernel(const float* __restrict__ U, const float* __restrict__ Vbb,
-                  float* __restrict__ P2, int b, int B) {
+                  __nv_bfloat16* __restrict__ P2, int b, int B) {
   using G = SimtGemm<64, 64, 16, 4, 4, false, false, float, float>;
   __shared__ float smem[G::SMEM_FLOATS];
   const int bb = blockIdx.z;
@@ -132,7 +134,16 @@ block_rows_kernel(const float* __restrict__ U, const float* __restrict__ Vbb,
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int gn = n0 + G::col_of(tx, j);
-      if (gn < N) P2[(int64_t)(j1 + gm) * b + j2 + gn] = acc[i][j];
+      if (gn < N) {
+        float v = acc[i][j];
+        __nv_bfloat16* o = P2 + (int64_t)(j1 + gm) * b + j2 + gn;
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl) {  // three bf16 planes of the fp32 value
+          const __nv_bfloat16 hb = __float2bfloat16_rn(v);
+          o[(int64_t)pl * b * b] = hb;
+          v -= __bfloat162float(hb);
+        }
+      }
     }
   }
 }
@@ -371,7 +382,8 @@ nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
 }
 
 __global__ void finish_block_kernel(SweepState* st, thanos_stats_t* stats, int64_t* r_ext,
-                                    long long nm_count, int is_nm) {
+                                    long long nm_count, int is_nm, const int32_t* tc_status) {
+  if (*tc_status != 0 && stats->status == 0) stats->status = *tc_status;
   unsigned long long cnt = is_nm ? (unsigned long long)nm_count : st->blk_count;
   if (!is_nm) {
     st->r -= (long long)cnt;
@@ -385,41 +397,6 @@ __global__ void finish_block_kernel(SweepState* st, thanos_stats_t* stats, int64
   stats->n_pruned += (long long)cnt;
   stats->n_blocks += 1;
   st->blk_count = 0;
-}
-
-// ------------------------------------------------------------------ W[:, j2:] += delta P2
-__global__ void __launch_bounds__(256)
-update_kernel(float* __restrict__ Wc, const float* __restrict__ D, const float* __restrict__ P2,
-              int c, int b, int j1, int Bw, int ldd) {
-  using G = SimtGemm<128, 128, 16, 8, 8, false, false, float, float>;
-  __shared__ float smem[G::SMEM_FLOATS];
-  const int j2 = j1 + Bw;
-  const int N = b - j2;
-  const int m0 = blockIdx.y * 128, n0 = blockIdx.x * 128;
-  float acc[8][8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-  G::run(D, ldd, P2 + (int64_t)j1 * b + j2, b, c, N, m0, n0, 0, Bw, acc, smem);
-  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    int gm = m0 + G::row_of(ty, i);
-    if (gm >= c) continue;
-#pragma unroll
-    for (int cj = 0; cj < 2; ++cj) {
-      int gn = n0 + G::col_of(tx, cj * 4);
-      if (gn >= N) continue;  // N and gn are multiples of 4
-      float4* wp = reinterpret_cast<float4*>(Wc + (int64_t)gm * b + j2 + gn);
-      float4 w = *wp;
-      w.x += acc[i][cj * 4 + 0];
-      w.y += acc[i][cj * 4 + 1];
-      w.z += acc[i][cj * 4 + 2];
-      w.w += acc[i][cj * 4 + 3];
-      *wp = w;
-    }
-  }
 }
 
 // ------------------------------------------------------------------ dtype conversion
@@ -450,12 +427,13 @@ __global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long lo
 
 struct SweepWs {
   float* Wc;   // fp32 working copy when the I/O dtype is not fp32
-  float* D;    // [c, B] change of the current block (delta)
+  __nv_bfloat16* D;    // [3][c, B] change of the current block (delta) as bf16 planes
   float* Ubb;  // [blocks, B, B] per-block matrices
   float* Vbb;
   float* G;
   float* S;
-  float* P2;   // [b, b]; rows of block j1..j2 hold V_bb U[j1:j2, j2:] in columns >= j2
+  __nv_bfloat16* P2;   // [3][b, b] bf16 planes; rows j1..j2 hold V_bb U[j1:j2, j2:] (columns >= j2)
+  int32_t* tc_status;  // device status word of the tensor-core products
   unsigned* hist;
   SweepState* st;
   unsigned* rowcnt;
@@ -469,12 +447,13 @@ bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, i
   Arena ar(workspace, ws_bytes);
   const size_t blocks = (size_t)ceil_div(b, B);
   w.Wc = need_wc ? ar.take<float>((size_t)c * b) : nullptr;
-  w.D = ar.take<float>((size_t)c * B);
+  w.D = ar.take<__nv_bfloat16>(3 * (size_t)c * B);
   w.Ubb = ar.take<float>(blocks * B * B);
   w.Vbb = ar.take<float>(blocks * B * B);
   w.G = ar.take<float>(blocks * B * B);
   w.S = ar.take<float>(blocks * B * B);
-  w.P2 = ar.take<float>((size_t)b * b);
+  w.P2 = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
+  w.tc_status = ar.take<int32_t>(4);
   w.hist = ar.take<unsigned>(HIST_BINS);
   w.st = ar.take<SweepState>(1);
   w.rowcnt = ar.take<unsigned>((size_t)c);
@@ -547,15 +526,31 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     THANOS_CHECK_LAUNCH();
   }
   THANOS_TRY(launch_block_solve(Wc, mask, w.G + (size_t)bb * B * B, w.S + (size_t)bb * B * B, B,
-                                w.D, c, b, j1, Bw, B, s_fixed, w.row_lists, w.list_counts, stats,
-                                stream));
+                                w.D, (int64_t)c * B, c, b, j1, Bw, B, s_fixed, w.row_lists,
+                                w.list_counts, stats, stream));
   if (j2 < b) {
-    dim3 g((unsigned)ceil_div(b - j2, 128), (unsigned)ceil_div(c, 128));
-    update_kernel<<<g, 256, 0, stream>>>(Wc, w.D, w.P2, c, b, j1, Bw, B);
-    THANOS_CHECK_LAUNCH();
+    // W[:, j2:] += delta P2[j1:j2, j2:]
+    TcGemmArgs g;
+    g.D = Wc + j2;
+    g.ldd = b;
+    g.A = w.D;
+    g.lda = B;
+    g.a_plane = (int64_t)c * B;
+    g.B = w.P2 + (int64_t)j1 * b + j2;
+    g.ldb = b;
+    g.b_plane = (int64_t)b * b;
+    g.b_kmajor = 0;
+    g.M = c;
+    g.N = b - j2;
+    g.K = Bw;
+    g.alpha = 1.f;
+    g.accumulate = 1;
+    g.status = w.tc_status;
+    THANOS_TRY(tc_gemm_split3(g, stream));
   }
   long long nm_count = mode == THANOS_NM ? (long long)c * (Bw / m) * n : 0;
-  finish_block_kernel<<<1, 1, 0, stream>>>(w.st, stats, r_ext, nm_count, mode == THANOS_NM);
+  finish_block_kernel<<<1, 1, 0, stream>>>(w.st, stats, r_ext, nm_count, mode == THANOS_NM,
+                                           w.tc_status);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
@@ -566,9 +561,9 @@ size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dty
   size_t t = 0;
   const size_t blocks = (size_t)ceil_div(b, B);
   if (dtype != THANOS_F32) t += round_up((size_t)c * b * sizeof(float), 256);
-  t += round_up((size_t)c * B * sizeof(float), 256);
+  t += round_up(3 * (size_t)c * B * sizeof(__nv_bfloat16), 256);
   t += 4 * round_up(blocks * B * B * sizeof(float), 256);
-  t += round_up((size_t)b * b * sizeof(float), 256);
+  t += round_up(3 * (size_t)b * b * sizeof(__nv_bfloat16), 256) + 256;
   t += round_up(HIST_BINS * sizeof(unsigned), 256);
   t += round_up(sizeof(SweepState), 256);
   t += round_up((size_t)c * sizeof(unsigned), 256);
@@ -604,6 +599,7 @@ thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b,
   if (!carve(w, workspace, ws_bytes, c, b, B, false)) return THANOS_ERR_WORKSPACE;
   THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
   THANOS_CUDA(cudaMemsetAsync(w.st, 0, sizeof(SweepState), stream));
+  THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
   return block_step(Wc, mask, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
                     stream);
@@ -634,6 +630,7 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
   if (mode == THANOS_UNSTRUCTURED) r = (long long)floor(p * (double)c * (double)b);
   init_sweep_kernel<<<1, 1, 0, stream>>>(w.st, stats, r);
   THANOS_CHECK_LAUNCH();
+  THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
   for (int64_t j1 = 0; j1 < b; j1 += B) {
     THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr, w,

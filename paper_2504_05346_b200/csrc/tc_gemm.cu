@@ -1,0 +1,440 @@
+// fp32-accurate GEMM on tcgen05: D = [D +] alpha * A * Bop with every operand given as three
+// bf16 planes (see tc_gemm.cuh).
+//
+// One persistent CTA per SM over 128 x 128 output tiles.  Roles:
+//   warp 0      TMA producer: per 64-wide k step the three planes of the A tile (128 rows x 64 k,
+//               K-major, 128-byte swizzle) and of the B tile (K-major: 128 n x 64 k; MN-major:
+//               two boxes of 64 n x 64 k) -- 96 KB per stage, two stages
+//   warp 1      tcgen05.mma issuer: per stage 6 plane pairs x 4 MMAs of 128 x 128 x 16
+//   warps 2..5  epilogue: TMEM -> registers -> D (fp32 read-modify-write) and, if asked, the
+//               result split into bf16 planes for the next product
+// TMEM: two 128 x 128 fp32 accumulators, so the epilogue of a tile overlaps the next tile's MMAs.
+// Every wait is bounded (see tc_common.cuh); on expiry the status word gets THANOS_ERR_TIMEOUT.
+#include "tc_gemm.cuh"
+
+#include "tc_common.cuh"
+
+namespace thanos {
+
+namespace {
+
+using namespace tc;
+
+constexpr int TM = 128;
+constexpr int TN = 128;
+constexpr int BK = 64;
+constexpr int STAGES = 2;
+constexpr int PLANE_TILE_BYTES = 128 * BK * 2;       // 16 KB: one plane of an operand tile
+constexpr int STAGE_BYTES = 6 * PLANE_TILE_BYTES;    // A planes 0..2, then B planes 0..2
+constexpr int B_OFFSET = 3 * PLANE_TILE_BYTES;
+constexpr int NTHREADS = 192;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr uint32_t TMEM_COLS = 256;
+
+struct Params {
+  float* D;
+  __nv_bfloat16* Dp;
+  int64_t ldd, d_batch, ldp, dp_plane, dp_batch;
+  int32_t* status;
+  int M, N, K, batch;
+  int tiles_m, tiles_n;
+  int b_kmajor, accumulate, upper_only;
+  float alpha;
+};
+
+// K-major operand tile: rows of 64 bf16 (128 bytes), 8 rows per 1024-byte swizzle atom.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading offset: not used by swizzled K-major layouts
+  d |= (uint64_t)(1024u >> 4) << 32;      // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                 // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+  return d;
+}
+// MN-major operand tile made of 64 n x 64 k boxes: a k row is 128 bytes, 8 k rows per atom, the
+// next 64 n are one box (8 KB) further.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(8192u >> 4) << 16;
+  d |= (uint64_t)(1024u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+__device__ __forceinline__ uint32_t make_idesc(int b_kmajor) {
+  uint32_t d = 0;
+  d |= 1u << 4;    // D fp32
+  d |= 1u << 7;    // A bf16
+  d |= 1u << 10;   // B bf16
+  if (!b_kmajor) d |= 1u << 16;  // B is MN-major (A is K-major: bit 15 clear)
+  d |= (uint32_t)(TN >> 3) << 17;
+  d |= (uint32_t)(TM >> 4) << 24;
+  return d;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int x, int y, int z, int w) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+      : "memory");
+}
+
+struct Tile {
+  int z, m0, n0;
+  bool skip;
+};
+__device__ __forceinline__ Tile decode_tile(const Params& p, int t) {
+  Tile r;
+  const int per = p.tiles_m * p.tiles_n;
+  r.z = t / per;
+  const int rem = t - r.z * per;
+  const int mi = rem / p.tiles_n;
+  r.m0 = mi * TM;
+  r.n0 = (rem - mi * p.tiles_n) * TN;
+  r.skip = p.upper_only && (r.n0 + TN - 1 < r.m0);
+  return r;
+}
+
+__constant__ int c_plane_a[6] = {0, 0, 1, 0, 2, 1};
+__constant__ int c_plane_b[6] = {0, 1, 0, 2, 0, 1};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+               const Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+  // bars[0..1] full, [2..3] empty, [4..5] tmem full, [6..7] tmem empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (2 + s); };
+  auto tfull_bar = [&](int q) { return bar_base + 8u * (4 + q); };
+  auto tempty_bar = [&](int q) { return bar_base + 8u * (6 + q); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int q = 0; q < 2; ++q) {
+      mbar_init(tfull_bar(q), 1);
+      mbar_init(tempty_bar(q), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_tiles = p.tiles_m * p.tiles_n * p.batch;
+  const int ksteps = (p.K + BK - 1) / BK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    int s = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const Tile tl = decode_tile(p, t);
+      if (tl.skip) continue;
+      for (int ks = 0; ks < ksteps && ok; ++ks) {
+        ok = mbar_wait(empty_bar(s), phase ^ 1u, abort_flag);
+        if (ok && lane == 0) {
+          const uint32_t dst = smem_base + (uint32_t)s * STAGE_BYTES;
+          const int k0 = ks * BK;
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+#pragma unroll
+          for (int pl = 0; pl < 3; ++pl)
+            tma_load_4d(dst + pl * PLANE_TILE_BYTES, &mapA, full_bar(s), k0, tl.m0, pl, tl.z);
+          if (p.b_kmajor) {
+#pragma unroll
+            for (int pl = 0; pl < 3; ++pl)
+              tma_load_4d(dst + B_OFFSET + pl * PLANE_TILE_BYTES, &mapB, full_bar(s), k0, tl.n0, pl,
+                          tl.z);
+          } else {
+#pragma unroll
+            for (int pl = 0; pl < 3; ++pl) {
+              tma_load_4d(dst + B_OFFSET + pl * PLANE_TILE_BYTES, &mapB, full_bar(s), tl.n0, k0, pl,
+                          tl.z);
+              tma_load_4d(dst + B_OFFSET + pl * PLANE_TILE_BYTES + 8192, &mapB, full_bar(s),
+                          tl.n0 + 64, k0, pl, tl.z);
+            }
+          }
+        }
+        __syncwarp();
+        if (++s == STAGES) {
+          s = 0;
+          phase ^= 1u;
+        }
+      }
+    }
+    // let copies that are still in flight land before the CTA's shared memory goes away
+    if (!ok) {
+      for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    const uint32_t idesc = make_idesc(p.b_kmajor);
+    int s = 0, q = 0;
+    uint32_t phase = 0, tphase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const Tile tl = decode_tile(p, t);
+      if (tl.skip) continue;
+      ok = mbar_wait(tempty_bar(q), tphase ^ 1u, abort_flag);
+      tc_fence_after();
+      for (int ks = 0; ks < ksteps && ok; ++ks) {
+        ok = mbar_wait(full_bar(s), phase, abort_flag);
+        tc_fence_after();
+        if (ok && lane == 0) {
+          const uint32_t sa = smem_base + (uint32_t)s * STAGE_BYTES;
+          const uint32_t sb = sa + B_OFFSET;
+#pragma unroll
+          for (int cb = 0; cb < 6; ++cb) {
+            const uint32_t pa = sa + (uint32_t)c_plane_a[cb] * PLANE_TILE_BYTES;
+            const uint32_t pb = sb + (uint32_t)c_plane_b[cb] * PLANE_TILE_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < BK / 16; ++k4) {
+              const uint64_t adesc = desc_kmajor(pa + k4 * 32);
+              const uint64_t bdesc =
+                  p.b_kmajor ? desc_kmajor(pb + k4 * 32) : desc_mnmajor(pb + k4 * 2048);
+              tc_mma_bf16(tmem_base + (uint32_t)q * TN, adesc, bdesc, idesc,
+                          (ks > 0 || cb > 0 || k4 > 0) ? 1u : 0u);
+            }
+          }
+          tc_commit(empty_bar(s));
+        }
+        __syncwarp();
+        if (++s == STAGES) {
+          s = 0;
+          phase ^= 1u;
+        }
+      }
+      if (ok && lane == 0) tc_commit(tfull_bar(q));
+      __syncwarp();
+      if (++q == 2) {
+        q = 0;
+        tphase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int g = warp & 3;  // TMEM lane quarter this warp may read
+    int q = 0;
+    uint32_t tphase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const Tile tl = decode_tile(p, t);
+      if (tl.skip) continue;
+      ok = mbar_wait(tfull_bar(q), tphase, abort_flag);
+      tc_fence_after();
+      if (ok) {
+        const int row = tl.m0 + 32 * g + lane;
+        float* drow = p.D ? p.D + (int64_t)tl.z * p.d_batch + (int64_t)row * p.ldd : nullptr;
+        __nv_bfloat16* prow =
+            p.Dp ? p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)row * p.ldp : nullptr;
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)q * TN;
+#pragma unroll 1
+        for (int cc = 0; cc < TN / 32; ++cc) {
+          uint32_t v[32];
+          tc_ld32(taddr + cc * 32, v);
+          tc_wait_ld();
+          if (row < p.M) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const int col = tl.n0 + cc * 32 + j;
+              if (col >= p.N) break;
+              float o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) o[e] = p.alpha * __uint_as_float(v[j + e]);
+              if (col + 3 < p.N) {
+                if (drow) {
+                  float4* dp4 = reinterpret_cast<float4*>(drow + col);
+                  if (p.accumulate) {
+                    const float4 old = *dp4;
+                    o[0] += old.x; o[1] += old.y; o[2] += old.z; o[3] += old.w;
+                  }
+                  *dp4 = make_float4(o[0], o[1], o[2], o[3]);
+                }
+                if (prow) {
+#pragma unroll
+                  for (int pl = 0; pl < 3; ++pl) {
+                    __nv_bfloat16 hb[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      hb[e] = __float2bfloat16_rn(o[e]);
+                      o[e] -= __bfloat162float(hb[e]);
+                    }
+                    uint2 pk;
+                    pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) |
+                           ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
+                    pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) |
+                           ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
+                    *reinterpret_cast<uint2*>(prow + (int64_t)pl * p.dp_plane + col) = pk;
+                  }
+                }
+              } else {
+                for (int e = 0; e < 4 && col + e < p.N; ++e) {
+                  float val = o[e];
+                  if (drow) {
+                    if (p.accumulate) val += drow[col + e];
+                    drow[col + e] = val;
+                  }
+                  if (prow) {
+                    for (int pl = 0; pl < 3; ++pl) {
+                      const __nv_bfloat16 hb = __float2bfloat16_rn(val);
+                      prow[(int64_t)pl * p.dp_plane + col + e] = hb;
+                      val -= __bfloat162float(hb);
+                    }
+                  }
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(q));
+      if (++q == 2) {
+        q = 0;
+        tphase ^= 1u;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(TMEM_COLS)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicCAS(p.status, 0, (int)THANOS_ERR_TIMEOUT);
+}
+
+bool make_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t inner, int64_t rows, int64_t ld,
+              int64_t plane_stride, int64_t batch, int64_t batch_stride, int box_inner,
+              int box_rows) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  if (plane_stride <= 0) plane_stride = ld;   // never stepped over when it has one entry
+  if (batch_stride <= 0) batch_stride = ld;
+  cuuint64_t gdim[4] = {(cuuint64_t)inner, (cuuint64_t)rows, 3, (cuuint64_t)batch};
+  cuuint64_t gstr[3] = {(cuuint64_t)ld * 2, (cuuint64_t)plane_stride * 2,
+                        (cuuint64_t)batch_stride * 2};
+  cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(base), gdim, gstr,
+             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__global__ void __launch_bounds__(256)
+split3_kernel(const float* __restrict__ X, int64_t ld, int64_t rows, int64_t cols,
+              __nv_bfloat16* __restrict__ planes, int64_t ldp, int64_t plane_stride) {
+  const int64_t q4 = cols >> 2;
+  const int64_t total = rows * q4;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    const int64_t r = e / q4;
+    const int64_t cq = e - r * q4;
+    const float4 x = *reinterpret_cast<const float4*>(X + r * ld + 4 * cq);
+    float o[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      __nv_bfloat16 hb[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        hb[k] = __float2bfloat16_rn(o[k]);
+        o[k] -= __bfloat162float(hb[k]);
+      }
+      uint2 pk;
+      pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) | ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
+      pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) | ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
+      *reinterpret_cast<uint2*>(planes + (int64_t)pl * plane_stride + r * ldp + 4 * cq) = pk;
+    }
+  }
+}
+
+}  // namespace
+
+thanos_status_t tc_gemm_split3(const TcGemmArgs& a, cudaStream_t stream) {
+  if (a.M <= 0 || a.N <= 0 || a.batch <= 0) return THANOS_OK;
+  if (a.K <= 0 || !a.A || !a.B || (!a.D && !a.Dp)) return THANOS_ERR_INVALID_ARG;
+  if (!aligned16(a.A) || !aligned16(a.B) || !aligned16(a.D) || !aligned16(a.Dp))
+    return THANOS_ERR_ALIGNMENT;
+  if (a.lda % 8 || a.ldb % 8 || a.a_plane % 8 || a.b_plane % 8 || a.a_batch % 8 || a.b_batch % 8)
+    return THANOS_ERR_ALIGNMENT;
+  if (a.D && (a.ldd % 4 || a.d_batch % 4)) return THANOS_ERR_ALIGNMENT;
+  if (a.Dp && (a.ldp % 4 || a.dp_plane % 4 || a.dp_batch % 4)) return THANOS_ERR_ALIGNMENT;
+  CUtensorMap mapA, mapB;
+  if (!make_map(&mapA, a.A, a.K, a.M, a.lda, a.a_plane, a.batch, a.a_batch, 64, 128))
+    return THANOS_ERR_CUDA;
+  const bool okb = a.b_kmajor
+                       ? make_map(&mapB, a.B, a.K, a.N, a.ldb, a.b_plane, a.batch, a.b_batch, 64, 128)
+                       : make_map(&mapB, a.B, a.N, a.K, a.ldb, a.b_plane, a.batch, a.b_batch, 64, 64);
+  if (!okb) return THANOS_ERR_CUDA;
+  Params p;
+  p.D = a.D;
+  p.Dp = a.Dp;
+  p.ldd = a.ldd;
+  p.d_batch = a.d_batch;
+  p.ldp = a.ldp;
+  p.dp_plane = a.dp_plane;
+  p.dp_batch = a.dp_batch;
+  p.status = a.status;
+  p.M = a.M;
+  p.N = a.N;
+  p.K = a.K;
+  p.batch = a.batch;
+  p.tiles_m = (a.M + TM - 1) / TM;
+  p.tiles_n = (a.N + TN - 1) / TN;
+  p.b_kmajor = a.b_kmajor;
+  p.accumulate = a.accumulate;
+  p.upper_only = a.upper_only;
+  p.alpha = a.alpha;
+  const long long tiles = (long long)p.tiles_m * p.tiles_n * p.batch;
+  if (tiles > (1ll << 30)) return THANOS_ERR_SHAPE;
+  const int G = sm_count();
+  const int grid = (int)(tiles < G ? tiles : G);
+  THANOS_CUDA(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)SMEM_BYTES));
+  tc_gemm_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+thanos_status_t split3_planes(const float* X, int64_t ld, int64_t rows, int64_t cols,
+                              __nv_bfloat16* planes, int64_t ldp, int64_t plane_stride,
+                              cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return THANOS_OK;
+  if (cols % 4 || ld % 4 || ldp % 4 || plane_stride % 4) return THANOS_ERR_ALIGNMENT;
+  int64_t blocks = ceil_div(rows * (cols / 4), 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  split3_kernel<<<(unsigned)blocks, 256, 0, stream>>>(X, ld, rows, cols, planes, ldp, plane_stride);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+}  // namespace thanos

@@ -497,3 +497,29 @@ def test_host_buffer_entry_point_matches_device_path(T):
     same = ~(Mh.numpy() != M.cpu().numpy()).any(axis=1)
     assert same.mean() >= 0.95
     assert PU.rel_fro(_np64(Wh)[same], _np64(Wp)[same]) <= 1e-3
+
+
+# ------------------------------------------------------------------------------ dense product
+@pytest.mark.parametrize("M,N,K,bt", [
+    (128, 128, 64, True), (128, 128, 64, False), (300, 520, 128, False), (300, 520, 128, True),
+    (64, 72, 8, False), (1000, 4096, 128, False), (257, 132, 200, True), (512, 384, 1024, True)])
+def test_dense_product_matches_float64(T, M, N, K, bt):
+    """The split-bf16 tensor-core product against a float64 product of the same fp32 inputs.
+    Bound: a few units of 2^-24 of sum |a||b| per 16-term tensor-core accumulation step."""
+    g = torch.Generator().manual_seed(M * 7 + N * 3 + K)
+    A = torch.randn((M, K), generator=g) * torch.exp(torch.randn((M, 1), generator=g))
+    Bm = torch.randn((N, K) if bt else (K, N), generator=g)
+    C0 = torch.randn((M, N), generator=g)
+    Ad, Bd = A.to(DEV), Bm.to(DEV)
+    want = _np64(A) @ (_np64(Bm).T if bt else _np64(Bm))
+    scale = np.abs(_np64(A)) @ np.abs(_np64(Bm).T if bt else _np64(Bm))
+    got = _np64(T.dense_product(Ad, Bd, b_transposed=bt))
+    assert np.max(np.abs(got - want) / scale) <= 3e-6
+    assert np.mean(np.abs(got - want) / scale) <= 4e-7
+    # accumulate with a scale factor, into a strided output
+    big = torch.zeros((M, N + 8), device=DEV)
+    big[:, :N] = C0.to(DEV)
+    T.dense_product(Ad, Bd, b_transposed=bt, alpha=-0.5, out=big[:, :N], accumulate=True)
+    got2 = _np64(big[:, :N])
+    assert np.max(np.abs(got2 - (_np64(C0) - 0.5 * want)) / (scale + np.abs(_np64(C0)))) <= 3e-6
+    assert float(big[:, N:].abs().max()) == 0.0
