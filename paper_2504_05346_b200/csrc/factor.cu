@@ -5,15 +5,19 @@
 //   column backwards), U = V^{-1} (upper).  Then H_d^{-1} = U^T U and, because V[j:, j:] is the
 //   same kind of factor of H_d[j:, j:], inv(H_d[j:, j:]) = U[j:, j:]^T U[j:, j:] for every j.
 //
-// Blocked right-looking factorisation with NB-wide panels (diagonal blocks in float64 inside
-// one CTA), then a divide-and-conquer triangular inverse whose levels are batched GEMMs.
+// Blocked right-looking factorisation with 128-wide panels: the 128 x 128 diagonal block is
+// factored and inverted by one CTA, the panel and the trailing update are tensor-core products
+// (three bf16 planes per operand, see tc_gemm.cuh); then a divide-and-conquer triangular inverse
+// whose levels are tensor-core products as well.
 #include "simt_gemm.cuh"
+#include "tc_gemm.cuh"
 
 namespace thanos {
 
 namespace {
 
-constexpr int NB = 64;
+constexpr int NB = 128;
+constexpr int DLD = NB + 4;  // row stride of the diagonal-block scratch (odd multiple of 16 bytes)
 
 // ---- mean(diag H) -> lambda, xnorm ---------------------------------------------------------
 __global__ void __launch_bounds__(1024)
@@ -50,263 +54,270 @@ __global__ void copy_damped_upper_kernel(const float* __restrict__ H, float* __r
   V[(int64_t)i * b + j] = v;
 }
 
-// ---- diagonal block: V22 V22^T = A22 (upper, reversed order) and its inverse, in float64 ----
-__global__ void __launch_bounds__(256)
-potrf_diag_kernel(float* __restrict__ V, int b, int k0, int n, float* __restrict__ Dinv,
-                  int32_t* __restrict__ status) {
-  extern __shared__ __align__(16) unsigned char potrf_smem[];
-  double (*S)[NB + 1] = reinterpret_cast<double (*)[NB + 1]>(potrf_smem);
-  double (*Si)[NB + 1] = S + NB;
+// ---- diagonal block: A22 = V22 V22^T (V22 upper, i.e. Cholesky from the last row backwards) and
+//      U22 = inv(V22).  One CTA, one thread per row.  With the rows and columns reversed this is
+//      an ordinary lower Cholesky L; n identity rows appended below the block turn into L^{-T}
+//      under the same elimination, which gives the inverse without a second pass.
+//      Left-looking in panels of 8 columns; every thread factors the 8 x 8 diagonal piece itself.
+__global__ void __launch_bounds__(2 * NB)
+diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* __restrict__ Up,
+                  int64_t plane, int b, int k0, int n, int32_t* __restrict__ status) {
+  extern __shared__ __align__(16) float dsm[];
+  float* L = dsm;                       // [2 n][DLD]
+  float* dblk = dsm + 2 * NB * DLD;     // [8][8]
   const int tid = threadIdx.x;
-  for (int e = tid; e < NB * NB; e += 256) {
-    int i = e / NB, j = e % NB;
-    double v = 0.0;
-    if (i < n && j < n) {
-      int a = i < j ? i : j, c = i < j ? j : i;
-      v = (double)V[(int64_t)(k0 + a) * b + k0 + c];
-    }
-    S[i][j] = v;
-    Si[i][j] = 0.0;
+  for (int e = tid; e < n * n; e += blockDim.x) {
+    const int i = e / n, j = e - i * n;
+    float v = 0.f;
+    if (j <= i) v = V[(int64_t)(k0 + n - 1 - i) * b + k0 + n - 1 - j];
+    L[i * DLD + j] = v;
+    L[(n + i) * DLD + j] = (i == j) ? 1.f : 0.f;
   }
   __syncthreads();
-  for (int k = n - 1; k >= 0; --k) {
-    double piv = S[k][k];
-    bool bad = !(piv > 0.0) || !isfinite(piv);
-    if (bad) {
-      if (tid == 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + k);
-      piv = 1.0;
+  const int r = tid;
+  const bool is_row = r < 2 * n;
+  float* Lr = L + (is_row ? r : 0) * DLD;
+  // identity row j is zero left of column j: its products start there (rounded down per warp)
+  const int first_nz = (r >= n) ? ((r - n) & ~31) : 0;
+  for (int c0 = 0; c0 < n; c0 += 8) {
+    const bool active = is_row && r >= c0;
+    float acc[8];
+    {
+      const float4 lo = *reinterpret_cast<const float4*>(Lr + c0);
+      const float4 hi = *reinterpret_cast<const float4*>(Lr + c0 + 4);
+      acc[0] = lo.x; acc[1] = lo.y; acc[2] = lo.z; acc[3] = lo.w;
+      acc[4] = hi.x; acc[5] = hi.y; acc[6] = hi.z; acc[7] = hi.w;
     }
-    double d = sqrt(piv);
-    __syncthreads();
-    if (tid == 0) S[k][k] = d;
-    for (int i = tid; i < k; i += 256) S[i][k] = S[i][k] / d;
-    __syncthreads();
-    // trailing (leading, in this order) update of the upper triangle i <= j < k
-    for (int e = tid; e < k * k; e += 256) {
-      int i = e / k, j = e % k;
-      if (i <= j) S[i][j] -= S[i][k] * S[j][k];
-    }
-    __syncthreads();
-  }
-  // inverse of the upper-triangular block, one column per thread (back substitution)
-  if (tid < n) {
-    const int cidx = tid;
-    for (int i = n - 1; i >= 0; --i) {
-      double x;
-      if (i > cidx) {
-        x = 0.0;
-      } else {
-        double acc = (i == cidx) ? 1.0 : 0.0;
-        for (int j = i + 1; j <= cidx; ++j) acc -= S[i][j] * Si[j][cidx];
-        x = acc / S[i][i];
+    if (active) {
+      const float* Pb = L + c0 * DLD;
+      for (int k = first_nz; k < c0; k += 4) {
+        const float4 av = *reinterpret_cast<const float4*>(Lr + k);
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const float4 bv = *reinterpret_cast<const float4*>(Pb + w * DLD + k);
+          acc[w] = fmaf(-av.x, bv.x, acc[w]);
+          acc[w] = fmaf(-av.y, bv.y, acc[w]);
+          acc[w] = fmaf(-av.z, bv.z, acc[w]);
+          acc[w] = fmaf(-av.w, bv.w, acc[w]);
+        }
       }
-      Si[i][cidx] = x;
     }
-  }
-  __syncthreads();
-  for (int e = tid; e < NB * NB; e += 256) {
-    int i = e / NB, j = e % NB;
-    if (i < n && j < n) {
-      if (j >= i) V[(int64_t)(k0 + i) * b + k0 + j] = (float)S[i][j];
-      Dinv[i * NB + j] = (j >= i) ? (float)Si[i][j] : 0.f;
-    } else {
-      Dinv[i * NB + j] = 0.f;
+    if (r >= c0 && r < c0 + 8) {
+#pragma unroll
+      for (int w = 0; w < 8; ++w) dblk[(r - c0) * 8 + w] = acc[w];
     }
-  }
-}
-
-// ---- panel: V12 = A12 * V22^{-T}, rows [0, k0), in place -----------------------------------
-__global__ void __launch_bounds__(256)
-trsm_panel_kernel(float* __restrict__ V, int b, int k0, int n, const float* __restrict__ Dinv) {
-  using G = SimtGemm<64, 64, 16, 4, 4, false, true, float, float>;
-  __shared__ float smem[G::SMEM_FLOATS];
-  float acc[4][4] = {};
-  int m0 = blockIdx.x * 64;
-  // out(m, j) = sum_k A12(m, k) * Dinv(j, k)
-  G::run(V + k0, b, Dinv, NB, k0, n, m0, 0, 0, n, acc, smem);
-  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
+    __syncthreads();
+    // 8 x 8 Cholesky of the diagonal piece, in registers, by every thread
+    float ld[8][8];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    int gm = m0 + G::row_of(ty, i);
-    if (gm >= k0) continue;
+    for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      int gn = G::col_of(tx, j);
-      if (gn < n) V[(int64_t)gm * b + k0 + gn] = acc[i][j];
+      for (int j = 0; j < 8; ++j) ld[i][j] = dblk[i * 8 + j];
+    float rinv[8];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      float d = ld[w][w];
+      if (!(d > 0.f) || !isfinite(d)) {
+        if (tid == 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + n - 1 - (c0 + w));
+        d = 1.f;
+      }
+      rinv[w] = 1.0f / sqrtf(d);
+#pragma unroll
+      for (int v = w; v < 8; ++v) ld[v][w] *= rinv[w];
+#pragma unroll
+      for (int v = w + 1; v < 8; ++v)
+#pragma unroll
+        for (int u = w + 1; u <= v; ++u) ld[v][u] = fmaf(-ld[v][w], ld[u][w], ld[v][u]);
     }
+    // this thread's row: x L_d^T = acc
+    float x[8];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      float t = acc[w];
+#pragma unroll
+      for (int v = 0; v < w; ++v) t = fmaf(-x[v], ld[w][v], t);
+      x[w] = t * rinv[w];
+    }
+    if (active) {
+      *reinterpret_cast<float4*>(Lr + c0) = make_float4(x[0], x[1], x[2], x[3]);
+      *reinterpret_cast<float4*>(Lr + c0 + 4) = make_float4(x[4], x[5], x[6], x[7]);
+    }
+    __syncthreads();
   }
-}
-
-// ---- trailing update: A11 -= V12 V12^T on upper-triangle tiles ------------------------------
-__global__ void __launch_bounds__(256)
-syrk_trailing_kernel(float* __restrict__ V, int b, int k0, int n, int nt) {
-  using G = SimtGemm<128, 128, 16, 8, 8, false, true, float, float>;
-  __shared__ float smem[G::SMEM_FLOATS];
-  int p = blockIdx.x, I = 0;
-  while (p >= nt - I) {
-    p -= nt - I;
-    ++I;
-  }
-  int J = I + p;
-  float acc[8][8];
+  // V22[i][j] = L[n-1-i][n-1-j];  U22[i][j] = inv(L)[n-1-i][n-1-j] = extra row (n-1-j), column n-1-i
+  for (int e = tid; e < n * n; e += blockDim.x) {
+    const int i = e / n, j = e - i * n;
+    float u = 0.f;
+    if (j >= i) {
+      V[(int64_t)(k0 + i) * b + k0 + j] = L[(n - 1 - i) * DLD + (n - 1 - j)];
+      u = L[(n + n - 1 - j) * DLD + (n - 1 - i)];
+    }
+    const int64_t o = (int64_t)(k0 + i) * b + k0 + j;
+    U[o] = u;
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-  G::run(V + k0, b, V + k0, b, k0, k0, I * 128, J * 128, 0, n, acc, smem);
-  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    int gm = I * 128 + G::row_of(ty, i);
-    if (gm >= k0) continue;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      int gn = J * 128 + G::col_of(tx, j);
-      if (gn < k0 && gn >= gm) V[(int64_t)gm * b + gn] -= acc[i][j];
+    for (int pl = 0; pl < 3; ++pl) {
+      const __nv_bfloat16 hb = __float2bfloat16_rn(u);
+      Up[(int64_t)pl * plane + o] = hb;
+      u -= __bfloat162float(hb);
     }
   }
 }
 
-// ---- U initialisation: inverted diagonal blocks, zero elsewhere -----------------------------
-__global__ void init_inverse_kernel(float* __restrict__ U, int b, const float* __restrict__ Dinv) {
-  int j = blockIdx.x * blockDim.x + threadIdx.x;
-  int i = blockIdx.y;
-  if (j >= b) return;
-  float v = 0.f;
-  if (i / NB == j / NB) v = Dinv[(int64_t)(i / NB) * NB * NB + (i % NB) * NB + (j % NB)];
-  U[(int64_t)i * b + j] = v;
+__global__ void fold_status_kernel(const int32_t* tc_status, int32_t* status) {
+  if (*tc_status != 0) atomicCAS(status, 0, *tc_status);
 }
 
-// Level of the divide-and-conquer inverse: for pair t with halves [r0, c0) and [c0, c0 + N):
-//   T = V12 * U22   (U22 upper: k <= n)        then        U12 = -U11 * T   (U11 upper: k >= m)
-template <int BT, int TT>
-__global__ void __launch_bounds__((BT / TT) * (BT / TT))
-trinv_gemm1_kernel(const float* __restrict__ V, const float* __restrict__ U,
-                   float* __restrict__ T, int b, int sz) {
-  using G = SimtGemm<BT, BT, 16, TT, TT, false, false, float, float>;
-  __shared__ float smem[G::SMEM_FLOATS];
-  int t = blockIdx.z;
-  int64_t r0 = (int64_t)2 * t * sz, c0 = r0 + sz;
-  if (c0 >= b) return;
-  int N = (int)((c0 + sz < b ? c0 + sz : b) - c0);
-  int m0 = blockIdx.y * BT, n0 = blockIdx.x * BT;
-  if (m0 >= sz || n0 >= N) return;
-  float acc[TT][TT];
-#pragma unroll
-  for (int i = 0; i < TT; ++i)
-#pragma unroll
-    for (int j = 0; j < TT; ++j) acc[i][j] = 0.f;
-  int kend = n0 + BT < N ? n0 + BT : N;
-  G::run(V + r0 * b + c0, b, U + c0 * b + c0, b, sz, N, m0, n0, 0, kend, acc, smem);
-  float* Tt = T + (int64_t)t * sz * sz;  // every pair before the last has N == sz
-  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
-#pragma unroll
-  for (int i = 0; i < TT; ++i) {
-    int gm = m0 + G::row_of(ty, i);
-    if (gm >= sz) continue;
-#pragma unroll
-    for (int j = 0; j < TT; ++j) {
-      int gn = n0 + G::col_of(tx, j);
-      if (gn < N) Tt[(int64_t)gm * N + gn] = acc[i][j];
-    }
-  }
-}
+struct PrepareWs {
+  float* V;
+  __nv_bfloat16* Vp;
+  __nv_bfloat16* Up;
+  __nv_bfloat16* Tp;
+  size_t t_elems;
+  float* lam;
+  int32_t* tc_status;
+};
 
-template <int BT, int TT>
-__global__ void __launch_bounds__((BT / TT) * (BT / TT))
-trinv_gemm2_kernel(float* __restrict__ U, const float* __restrict__ T, int b, int sz) {
-  using G = SimtGemm<BT, BT, 16, TT, TT, false, false, float, float>;
-  __shared__ float smem[G::SMEM_FLOATS];
-  int t = blockIdx.z;
-  int64_t r0 = (int64_t)2 * t * sz, c0 = r0 + sz;
-  if (c0 >= b) return;
-  int N = (int)((c0 + sz < b ? c0 + sz : b) - c0);
-  int m0 = blockIdx.y * BT, n0 = blockIdx.x * BT;
-  if (m0 >= sz || n0 >= N) return;
-  float acc[TT][TT];
-#pragma unroll
-  for (int i = 0; i < TT; ++i)
-#pragma unroll
-    for (int j = 0; j < TT; ++j) acc[i][j] = 0.f;
-  const float* Tt = T + (int64_t)t * sz * sz;
-  G::run(U + r0 * b + r0, b, Tt, N, sz, N, m0, n0, m0, sz, acc, smem);
-  const int tx = threadIdx.x % G::TX, ty = threadIdx.x / G::TX;
-#pragma unroll
-  for (int i = 0; i < TT; ++i) {
-    int gm = m0 + G::row_of(ty, i);
-    if (gm >= sz) continue;
-#pragma unroll
-    for (int j = 0; j < TT; ++j) {
-      int gn = n0 + G::col_of(tx, j);
-      if (gn < N) U[(r0 + gm) * b + c0 + gn] = -acc[i][j];
-    }
-  }
+size_t t_plane_elems(int64_t b) { return (size_t)b * b / 4 + (size_t)b * NB + 64; }
+
+bool carve_prepare(PrepareWs& w, void* workspace, size_t ws_bytes, int64_t b) {
+  Arena ar(workspace, ws_bytes);
+  w.V = ar.take<float>((size_t)b * b);
+  w.Vp = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
+  w.Up = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
+  w.t_elems = round_up(t_plane_elems(b), 64);
+  w.Tp = ar.take<__nv_bfloat16>(3 * w.t_elems);
+  w.lam = ar.take<float>(1);
+  w.tc_status = ar.take<int32_t>(4);
+  return ar.ok();
 }
 
 }  // namespace
 
 size_t prepare_workspace_bytes(int64_t b) {
-  size_t nblk = (size_t)ceil_div(b, NB);
-  size_t v = round_up((size_t)b * b * sizeof(float), 256);
-  size_t d = round_up(nblk * NB * NB * sizeof(float), 256);
-  size_t t = round_up(((size_t)b * b / 4 + (size_t)b * NB) * sizeof(float), 256);
-  return v + d + t + 256;
+  size_t t = round_up((size_t)b * b * sizeof(float), 256);
+  t += 2 * round_up(3 * (size_t)b * b * sizeof(__nv_bfloat16), 256);
+  t += round_up(3 * round_up(t_plane_elems(b), 64) * sizeof(__nv_bfloat16), 256);
+  return t + 3 * 256;
 }
 
 thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel, float* factor,
                                      float* xnorm, void* workspace, size_t ws_bytes,
                                      int32_t* status_dev, cudaStream_t stream) {
   const int b = (int)b64;
-  Arena ar(workspace, ws_bytes);
-  int nblk = (int)ceil_div(b, NB);
-  float* V = ar.take<float>((size_t)b * b);
-  float* Dinv = ar.take<float>((size_t)nblk * NB * NB);
-  float* T = ar.take<float>((size_t)b * b / 4 + (size_t)b * NB);
-  float* lam = ar.take<float>(1);
-  if (!ar.ok()) return THANOS_ERR_WORKSPACE;
+  PrepareWs w;
+  if (!carve_prepare(w, workspace, ws_bytes, b)) return THANOS_ERR_WORKSPACE;
+  const int64_t plane = (int64_t)b * b;
+  const int nblk = (int)ceil_div(b, NB);
 
-  diag_stats_kernel<<<1, 1024, 0, stream>>>(H, b, damp_rel, xnorm, lam);
+  diag_stats_kernel<<<1, 1024, 0, stream>>>(H, b, damp_rel, xnorm, w.lam);
   THANOS_CHECK_LAUNCH();
   dim3 cg((unsigned)ceil_div(b, 256), (unsigned)b);
-  copy_damped_upper_kernel<<<cg, 256, 0, stream>>>(H, V, b, lam);
+  copy_damped_upper_kernel<<<cg, 256, 0, stream>>>(H, w.V, b, w.lam);
   THANOS_CHECK_LAUNCH();
+  THANOS_CUDA(cudaMemsetAsync(factor, 0, (size_t)plane * sizeof(float), stream));
+  THANOS_CUDA(cudaMemsetAsync(w.Up, 0, 3 * (size_t)plane * sizeof(__nv_bfloat16), stream));
+  THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
 
-  constexpr int POTRF_SMEM = 2 * NB * (NB + 1) * (int)sizeof(double);
-  THANOS_CUDA(cudaFuncSetAttribute(potrf_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   POTRF_SMEM));
+  constexpr int DIAG_SMEM = (2 * NB * DLD + 64) * (int)sizeof(float);
+  THANOS_CUDA(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   DIAG_SMEM));
+  // ---- H_d = V V^T, panels from the last one backwards
   for (int kb = nblk - 1; kb >= 0; --kb) {
-    int k0 = kb * NB;
-    int n = (b - k0 < NB) ? b - k0 : NB;
-    float* Dk = Dinv + (size_t)kb * NB * NB;
-    potrf_diag_kernel<<<1, 256, POTRF_SMEM, stream>>>(V, b, k0, n, Dk, status_dev);
+    const int k0 = kb * NB;
+    const int n = (b - k0 < NB) ? b - k0 : NB;
+    diag_block_kernel<<<1, 2 * NB, DIAG_SMEM, stream>>>(w.V, factor, w.Up, plane, b, k0, n,
+                                                       status_dev);
     THANOS_CHECK_LAUNCH();
-    if (k0 > 0) {
-      trsm_panel_kernel<<<(unsigned)ceil_div(k0, 64), 256, 0, stream>>>(V, b, k0, n, Dk);
-      THANOS_CHECK_LAUNCH();
-      int nt = (int)ceil_div(k0, 128);
-      syrk_trailing_kernel<<<nt * (nt + 1) / 2, 256, 0, stream>>>(V, b, k0, n, nt);
-      THANOS_CHECK_LAUNCH();
-    }
+    if (k0 == 0) break;
+    // V12 = A12 U22^T (rows above the block), written over A12 and as planes
+    THANOS_TRY(split3_planes(w.V + k0, b, k0, n, w.Vp + k0, b, plane, stream));
+    TcGemmArgs g;
+    g.D = w.V + k0;
+    g.ldd = b;
+    g.Dp = w.Vp + k0;
+    g.ldp = b;
+    g.dp_plane = plane;
+    g.A = w.Vp + k0;
+    g.lda = b;
+    g.a_plane = plane;
+    g.B = w.Up + (int64_t)k0 * b + k0;
+    g.ldb = b;
+    g.b_plane = plane;
+    g.b_kmajor = 1;
+    g.M = k0;
+    g.N = n;
+    g.K = n;
+    g.status = w.tc_status;
+    THANOS_TRY(tc_gemm_split3(g, stream));
+    // A11 -= V12 V12^T on the tiles that touch the upper triangle
+    TcGemmArgs y;
+    y.D = w.V;
+    y.ldd = b;
+    y.A = w.Vp + k0;
+    y.lda = b;
+    y.a_plane = plane;
+    y.B = w.Vp + k0;
+    y.ldb = b;
+    y.b_plane = plane;
+    y.b_kmajor = 1;
+    y.M = k0;
+    y.N = k0;
+    y.K = n;
+    y.alpha = -1.f;
+    y.accumulate = 1;
+    y.upper_only = 1;
+    y.status = w.tc_status;
+    THANOS_TRY(tc_gemm_split3(y, stream));
   }
 
-  init_inverse_kernel<<<cg, 256, 0, stream>>>(factor, b, Dinv);
-  THANOS_CHECK_LAUNCH();
+  // ---- U = inv(V) by halves: for the pair of diagonal blocks [r0, c0) and [c0, c0 + N),
+  //      U12 = -U11 (V12 U22)
   for (int64_t sz = NB; sz < b; sz *= 2) {
-    int npairs = (int)ceil_div(b, 2 * sz);
-    if (sz <= 64) {
-      dim3 g((unsigned)ceil_div(sz, 64), (unsigned)ceil_div(sz, 64), (unsigned)npairs);
-      trinv_gemm1_kernel<64, 4><<<g, 256, 0, stream>>>(V, factor, T, b, (int)sz);
-      THANOS_CHECK_LAUNCH();
-      trinv_gemm2_kernel<64, 4><<<g, 256, 0, stream>>>(factor, T, b, (int)sz);
-      THANOS_CHECK_LAUNCH();
-    } else {
-      dim3 g((unsigned)ceil_div(sz, 128), (unsigned)ceil_div(sz, 128), (unsigned)npairs);
-      trinv_gemm1_kernel<128, 8><<<g, 256, 0, stream>>>(V, factor, T, b, (int)sz);
-      THANOS_CHECK_LAUNCH();
-      trinv_gemm2_kernel<128, 8><<<g, 256, 0, stream>>>(factor, T, b, (int)sz);
-      THANOS_CHECK_LAUNCH();
+    const int npairs = (int)ceil_div(b, 2 * sz);
+    for (int t = 0; t < npairs; ++t) {
+      const int64_t r0 = 2 * t * sz, c0 = r0 + sz;
+      if (c0 >= b) break;
+      const int N = (int)((c0 + sz < b ? c0 + sz : b) - c0);
+      __nv_bfloat16* Tt = w.Tp + (size_t)t * sz * sz;
+      TcGemmArgs g;
+      g.Dp = Tt;
+      g.ldp = N;
+      g.dp_plane = (int64_t)w.t_elems;
+      g.A = w.Vp + r0 * b + c0;
+      g.lda = b;
+      g.a_plane = plane;
+      g.B = w.Up + c0 * b + c0;
+      g.ldb = b;
+      g.b_plane = plane;
+      g.b_kmajor = 0;
+      g.M = (int)sz;
+      g.N = N;
+      g.K = N;
+      g.status = w.tc_status;
+      THANOS_TRY(tc_gemm_split3(g, stream));
+      TcGemmArgs h;
+      h.D = factor + r0 * b + c0;
+      h.ldd = b;
+      h.Dp = w.Up + r0 * b + c0;
+      h.ldp = b;
+      h.dp_plane = plane;
+      h.A = w.Up + r0 * b + r0;
+      h.lda = b;
+      h.a_plane = plane;
+      h.B = Tt;
+      h.ldb = N;
+      h.b_plane = (int64_t)w.t_elems;
+      h.b_kmajor = 0;
+      h.M = (int)sz;
+      h.N = N;
+      h.K = (int)sz;
+      h.alpha = -1.f;
+      h.status = w.tc_status;
+      THANOS_TRY(tc_gemm_split3(h, stream));
     }
   }
+  fold_status_kernel<<<1, 1, 0, stream>>>(w.tc_status, status_dev);
+  THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
 

@@ -6,7 +6,7 @@
 //               K-major, 128-byte swizzle) and of the B tile (K-major: 128 n x 64 k; MN-major:
 //               two boxes of 64 n x 64 k) -- 96 KB per stage, two stages
 //   warp 1      tcgen05.mma issuer: per stage 6 plane pairs x 4 MMAs of 128 x 128 x 16
-//   warps 2..5  epilogue: TMEM -> registers -> D (fp32 read-modify-write) and, if asked, the
+//   warps 2..9  epilogue: TMEM -> registers -> D (fp32 read-modify-write) and, if asked, the
 //               result split into bf16 planes for the next product
 // TMEM: two 128 x 128 fp32 accumulators, so the epilogue of a tile overlaps the next tile's MMAs.
 // Every wait is bounded (see tc_common.cuh); on expiry the status word gets THANOS_ERR_TIMEOUT.
@@ -27,7 +27,7 @@ constexpr int STAGES = 2;
 constexpr int PLANE_TILE_BYTES = 128 * BK * 2;       // 16 KB: one plane of an operand tile
 constexpr int STAGE_BYTES = 6 * PLANE_TILE_BYTES;    // A planes 0..2, then B planes 0..2
 constexpr int B_OFFSET = 3 * PLANE_TILE_BYTES;
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 320;
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 256;
 
@@ -129,7 +129,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     }
     for (int q = 0; q < 2; ++q) {
       mbar_init(tfull_bar(q), 1);
-      mbar_init(tempty_bar(q), 4);
+      mbar_init(tempty_bar(q), 8);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -238,43 +238,52 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------ epilogue
-    const int g = warp & 3;  // TMEM lane quarter this warp may read
+    // Warp w reads TMEM lanes 32 (w & 3) .. +31 (one output row per thread) and the column half
+    // (w - 2) / 4.  The old values of D are fetched before the accumulator is waited for, so
+    // their latency overlaps the tile's MMAs.
+    const int g = warp & 3;
+    const int h = (warp - 2) >> 2;
     int q = 0;
     uint32_t tphase = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       const Tile tl = decode_tile(p, t);
       if (tl.skip) continue;
+      const int row = tl.m0 + 32 * g + lane;
+      const int cbase = tl.n0 + 64 * h;
+      float* drow = p.D ? p.D + (int64_t)tl.z * p.d_batch + (int64_t)row * p.ldd : nullptr;
+      __nv_bfloat16* prow =
+          p.Dp ? p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)row * p.ldp : nullptr;
+      const bool full = row < p.M && cbase + 63 < p.N;  // whole 64-column strip inside D
+      float4 old[16];
+      if (full && drow && p.accumulate) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) old[j] = *reinterpret_cast<const float4*>(drow + cbase + 4 * j);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) old[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
       ok = mbar_wait(tfull_bar(q), tphase, abort_flag);
       tc_fence_after();
       if (ok) {
-        const int row = tl.m0 + 32 * g + lane;
-        float* drow = p.D ? p.D + (int64_t)tl.z * p.d_batch + (int64_t)row * p.ldd : nullptr;
-        __nv_bfloat16* prow =
-            p.Dp ? p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)row * p.ldp : nullptr;
-        const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)q * TN;
-#pragma unroll 1
-        for (int cc = 0; cc < TN / 32; ++cc) {
+        const uint32_t taddr =
+            tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)q * TN + (uint32_t)h * 64;
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
           uint32_t v[32];
           tc_ld32(taddr + cc * 32, v);
           tc_wait_ld();
           if (row < p.M) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-              const int col = tl.n0 + cc * 32 + j;
-              if (col >= p.N) break;
+              const int col = cbase + cc * 32 + j;
               float o[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) o[e] = p.alpha * __uint_as_float(v[j + e]);
-              if (col + 3 < p.N) {
-                if (drow) {
-                  float4* dp4 = reinterpret_cast<float4*>(drow + col);
-                  if (p.accumulate) {
-                    const float4 old = *dp4;
-                    o[0] += old.x; o[1] += old.y; o[2] += old.z; o[3] += old.w;
-                  }
-                  *dp4 = make_float4(o[0], o[1], o[2], o[3]);
-                }
+              if (full) {
+                const float4 od = old[cc * 8 + (j >> 2)];
+                o[0] += od.x; o[1] += od.y; o[2] += od.z; o[3] += od.w;
+                if (drow) *reinterpret_cast<float4*>(drow + col) = make_float4(o[0], o[1], o[2], o[3]);
                 if (prow) {
 #pragma unroll
                   for (int pl = 0; pl < 3; ++pl) {
