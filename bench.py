@@ -29,7 +29,7 @@ import workloads as WL
 
 METRIC = "pruned_weights_per_sec"
 UNIT = "weights/s"
-TOKEN_CHUNK = 32768  # tokens per thanos_hessian_accumulate call
+TOKEN_CHUNK = 262144  # tokens per thanos_hessian_accumulate call (the activations are resident)
 
 
 def _peaks():
