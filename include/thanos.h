@@ -192,7 +192,7 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
  * (every GPU that loads the library holds it until the process exits).  The call allocates
  * nothing and frees nothing.  A layer fits when
  *     thanos_workspace_bytes(THANOS_WS_PRUNE, c, b, B, wdtype) <= 4 MiB
- * (for example 512 x 512 fp32 with B = 128, or 256 x 1024 bf16 with B = 64); anything larger
+ * (for example 512 x 512 fp32 or 256 x 512 bf16 with B = 128); anything larger
  * is refused with THANOS_ERR_WORKSPACE before any work is enqueued.
  *
  * The first call on a device looks up the device address of that array (once per device, with
