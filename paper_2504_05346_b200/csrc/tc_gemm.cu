@@ -6,8 +6,9 @@
 //               K-major, 128-byte swizzle) and of the B tile (K-major: 128 n x 64 k; MN-major:
 //               two boxes of 64 n x 64 k) -- 96 KB per stage, two stages
 //   warp 1      tcgen05.mma issuer: per stage 6 plane pairs x 4 MMAs of 128 x 128 x 16
-//   warps 2..9  epilogue: TMEM -> registers -> D (fp32 read-modify-write) and, if asked, the
-//               result split into bf16 planes for the next product
+//   warps 2..9  epilogue: TMEM -> registers -> 128 x 32 fp32 staging buffers in shared memory ->
+//               TMA reduce-add (or store) into D; if asked, the result also split into bf16
+//               planes for the next product
 // TMEM: two 128 x 128 fp32 accumulators, so the epilogue of a tile overlaps the next tile's MMAs.
 // Every wait is bounded (see tc_common.cuh); on expiry the status word gets THANOS_ERR_TIMEOUT.
 #include "tc_gemm.cuh"
@@ -28,7 +29,9 @@ constexpr int PLANE_TILE_BYTES = 128 * BK * 2;       // 16 KB: one plane of an o
 constexpr int STAGE_BYTES = 6 * PLANE_TILE_BYTES;    // A planes 0..2, then B planes 0..2
 constexpr int B_OFFSET = 3 * PLANE_TILE_BYTES;
 constexpr int NTHREADS = 320;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int STAGING_BYTES = 128 * 32 * 4;          // 16 KB: 128 rows x 32 fp32 columns of D
+constexpr size_t SMEM_BYTES =
+    (size_t)STAGES * STAGE_BYTES + 2 * STAGING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 256;
 
 struct Params {
@@ -83,6 +86,26 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int x,
+                                                  int y, int z) {
+  asm volatile(
+      "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::
+          "l"(reinterpret_cast<uint64_t>(map)),
+      "r"(src), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y,
+                                             int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+          reinterpret_cast<uint64_t>(map)),
+      "r"(src), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 struct Tile {
   int z, m0, n0;
   bool skip;
@@ -104,11 +127,12 @@ __constant__ int c_plane_b[6] = {0, 1, 0, 2, 0, 1};
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-               const Params p) {
+               const __grid_constant__ CUtensorMap mapD, const Params p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+  uint64_t* bars =
+      reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES + 2 * STAGING_BYTES);
   // bars[0..1] full, [2..3] empty, [4..5] tmem full, [6..7] tmem empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
@@ -239,81 +263,93 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   } else {
     // ------------------------------------------------------------ epilogue
     // Warp w reads TMEM lanes 32 (w & 3) .. +31 (one output row per thread) and the column half
-    // (w - 2) / 4.  The old values of D are fetched before the accumulator is waited for, so
-    // their latency overlaps the tile's MMAs.
+    // h = (w - 2) / 4, 32 columns at a time.  The four warps of a half share one 128 x 32 fp32
+    // staging buffer (128-byte swizzle); one thread of the half hands it to TMA, which adds it to
+    // D (or stores it) with full-line accesses and no read in the SM.
     const int g = warp & 3;
     const int h = (warp - 2) >> 2;
+    const bool issuer = g == 0 && lane == 0;
+    unsigned char* stg = smem + (size_t)STAGES * STAGE_BYTES + (size_t)h * STAGING_BYTES;
+    const uint32_t stg_addr = smem_u32(stg);
+    const int r_in_tile = 32 * g + lane;
     int q = 0;
     uint32_t tphase = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+    // After a failed wait the warp keeps walking the tiles (the waits then return at once) so
+    // that the four warps of a half always meet at the same named barriers.
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
       const Tile tl = decode_tile(p, t);
       if (tl.skip) continue;
-      const int row = tl.m0 + 32 * g + lane;
-      const int cbase = tl.n0 + 64 * h;
-      float* drow = p.D ? p.D + (int64_t)tl.z * p.d_batch + (int64_t)row * p.ldd : nullptr;
+      const int row = tl.m0 + r_in_tile;
       __nv_bfloat16* prow =
           p.Dp ? p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)row * p.ldp : nullptr;
-      const bool full = row < p.M && cbase + 63 < p.N;  // whole 64-column strip inside D
-      float4 old[16];
-      if (full && drow && p.accumulate) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) old[j] = *reinterpret_cast<const float4*>(drow + cbase + 4 * j);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) old[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-      ok = mbar_wait(tfull_bar(q), tphase, abort_flag);
+      ok = ok && mbar_wait(tfull_bar(q), tphase, abort_flag);
       tc_fence_after();
-      if (ok) {
+      {
         const uint32_t taddr =
             tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)q * TN + (uint32_t)h * 64;
-#pragma unroll
+#pragma unroll 1
         for (int cc = 0; cc < 2; ++cc) {
           uint32_t v[32];
-          tc_ld32(taddr + cc * 32, v);
-          tc_wait_ld();
-          if (row < p.M) {
+          if (ok) {
+            tc_ld32(taddr + cc * 32, v);
+            tc_wait_ld();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0u;
+          }
+          const int cbase = tl.n0 + 64 * h + 32 * cc;
+          if (p.D) {
+            // the buffer is free once TMA has read the previous chunk out of it
+            if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            named_bar_sync(1 + 2 * h, 128);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 o;
+              o.x = p.alpha * __uint_as_float(v[4 * j + 0]);
+              o.y = p.alpha * __uint_as_float(v[4 * j + 1]);
+              o.z = p.alpha * __uint_as_float(v[4 * j + 2]);
+              o.w = p.alpha * __uint_as_float(v[4 * j + 3]);
+              *reinterpret_cast<float4*>(stg + r_in_tile * 128 + ((j ^ (r_in_tile & 7)) << 4)) = o;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            named_bar_sync(2 + 2 * h, 128);
+            if (issuer && ok && cbase < p.N) {
+              if (p.accumulate) tma_reduce_add_3d(&mapD, stg_addr, cbase, tl.m0, tl.z);
+              else tma_store_3d(&mapD, stg_addr, cbase, tl.m0, tl.z);
+              asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+          }
+          if (prow && ok && row < p.M) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-              const int col = cbase + cc * 32 + j;
+              const int col = cbase + j;
               float o[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) o[e] = p.alpha * __uint_as_float(v[j + e]);
-              if (full) {
-                const float4 od = old[cc * 8 + (j >> 2)];
-                o[0] += od.x; o[1] += od.y; o[2] += od.z; o[3] += od.w;
-                if (drow) *reinterpret_cast<float4*>(drow + col) = make_float4(o[0], o[1], o[2], o[3]);
-                if (prow) {
+              if (col + 3 < p.N) {
 #pragma unroll
-                  for (int pl = 0; pl < 3; ++pl) {
-                    __nv_bfloat16 hb[4];
+                for (int pl = 0; pl < 3; ++pl) {
+                  __nv_bfloat16 hb[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                      hb[e] = __float2bfloat16_rn(o[e]);
-                      o[e] -= __bfloat162float(hb[e]);
-                    }
-                    uint2 pk;
-                    pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) |
-                           ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
-                    pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) |
-                           ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
-                    *reinterpret_cast<uint2*>(prow + (int64_t)pl * p.dp_plane + col) = pk;
+                  for (int e = 0; e < 4; ++e) {
+                    hb[e] = __float2bfloat16_rn(o[e]);
+                    o[e] -= __bfloat162float(hb[e]);
                   }
+                  uint2 pk;
+                  pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) |
+                         ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
+                  pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) |
+                         ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
+                  *reinterpret_cast<uint2*>(prow + (int64_t)pl * p.dp_plane + col) = pk;
                 }
               } else {
                 for (int e = 0; e < 4 && col + e < p.N; ++e) {
                   float val = o[e];
-                  if (drow) {
-                    if (p.accumulate) val += drow[col + e];
-                    drow[col + e] = val;
-                  }
-                  if (prow) {
-                    for (int pl = 0; pl < 3; ++pl) {
-                      const __nv_bfloat16 hb = __float2bfloat16_rn(val);
-                      prow[(int64_t)pl * p.dp_plane + col + e] = hb;
-                      val -= __bfloat162float(hb);
-                    }
+                  for (int pl = 0; pl < 3; ++pl) {
+                    const __nv_bfloat16 hb = __float2bfloat16_rn(val);
+                    prow[(int64_t)pl * p.dp_plane + col + e] = hb;
+                    val -= __bfloat162float(hb);
                   }
                 }
               }
@@ -329,6 +365,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         tphase ^= 1u;
       }
     }
+    // every bulk store of this thread has to be complete before the kernel ends
+    if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   tc_fence_before();
@@ -404,6 +442,20 @@ thanos_status_t tc_gemm_split3(const TcGemmArgs& a, cudaStream_t stream) {
                        ? make_map(&mapB, a.B, a.K, a.N, a.ldb, a.b_plane, a.batch, a.b_batch, 64, 128)
                        : make_map(&mapB, a.B, a.N, a.K, a.ldb, a.b_plane, a.batch, a.b_batch, 64, 64);
   if (!okb) return THANOS_ERR_CUDA;
+  CUtensorMap mapD = mapA;  // placeholder when no fp32 output is requested
+  if (a.D) {
+    EncodeTiledFn enc = encode_fn();
+    const int64_t dbs = a.d_batch > 0 ? a.d_batch : a.ldd;
+    cuuint64_t gdim[3] = {(cuuint64_t)a.N, (cuuint64_t)a.M, (cuuint64_t)a.batch};
+    cuuint64_t gstr[2] = {(cuuint64_t)a.ldd * 4, (cuuint64_t)dbs * 4};
+    cuuint32_t box[3] = {32, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (!enc || enc(&mapD, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, a.D, gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return THANOS_ERR_CUDA;
+  }
   Params p;
   p.D = a.D;
   p.Dp = a.Dp;
@@ -429,7 +481,7 @@ thanos_status_t tc_gemm_split3(const TcGemmArgs& a, cudaStream_t stream) {
   const int grid = (int)(tiles < G ? tiles : G);
   THANOS_CUDA(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)SMEM_BYTES));
-  tc_gemm_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
+  tc_gemm_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(mapA, mapB, mapD, p);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
