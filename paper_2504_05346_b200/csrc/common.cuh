@@ -33,6 +33,20 @@ inline void count_launch(int n = 1) { g_launch_count.fetch_add(n, std::memory_or
     if (st__ != THANOS_OK) return st__;                     \
   } while (0)
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per device and call site instead of once
+// per launch (`done` is the call site's static bit set, one bit per device).
+template <typename F>
+inline cudaError_t ensure_max_dyn_smem(F func, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_relaxed) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_relaxed);
+  return e;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

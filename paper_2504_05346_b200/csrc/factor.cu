@@ -219,8 +219,10 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
   THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
 
   constexpr int DIAG_SMEM = (2 * NB * DLD + 64) * (int)sizeof(float);
-  THANOS_CUDA(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   DIAG_SMEM));
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(diag_block_kernel, DIAG_SMEM, done));
+  }
   // ---- H_d = V V^T, panels from the last one backwards
   for (int kb = nblk - 1; kb >= 0; --kb) {
     const int k0 = kb * NB;

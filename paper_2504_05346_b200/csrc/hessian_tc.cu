@@ -381,8 +381,10 @@ thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld
   }
   long long units = (long long)p.n_tiles * p.n_slices;
   int grid = (int)(units < G ? units : G);
-  THANOS_CUDA(cudaFuncSetAttribute(hessian_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)SMEM_BYTES));
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(hessian_tc_kernel, (int)SMEM_BYTES, done));
+  }
   hessian_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(tmap, p);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;

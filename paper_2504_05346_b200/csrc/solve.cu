@@ -552,9 +552,10 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
   if (warps < 1) return THANOS_ERR_SHAPE;
   if (warps > 12) warps = 12;
   const size_t smem = 4 * (size_t)lay.mat_floats + (size_t)warps * lay.per_warp_bytes;
-  THANOS_CUDA(cudaFuncSetAttribute(solve_rows_fast_kernel<NR>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)SOLVE_SMEM_BUDGET));
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_fast_kernel<NR>, (int)SOLVE_SMEM_BUDGET, done));
+  }
   int64_t grid = ceil_div(c, warps);
   if (grid > 148) grid = 148;
   solve_rows_fast_kernel<NR><<<(unsigned)grid, warps * 32, smem, stream>>>(
@@ -568,7 +569,7 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
 
 // Largest system the general kernel can hold for one warp.
 bool solve_supported(int s_direct_max, int n_small_max) {
-  if (n_small_max + 1 <= 96) return true;
+  if (n_small_max + 1 <= 160) return true;
   return general_per_warp_bytes(s_direct_max) <= SOLVE_SMEM_BUDGET;
 }
 
@@ -583,15 +584,16 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
                                    thanos_stats_t* stats, cudaStream_t stream) {
   const bool uniform = s_fixed >= 0;
   const int n_small = uniform ? (s_fixed < Bw - s_fixed ? s_fixed : Bw - s_fixed) : Bw / 2;
-  if (n_small + 1 > 96) {
+  if (n_small + 1 > 160) {
     const int smax = uniform ? s_fixed : Bw;
     size_t per_warp = general_per_warp_bytes(smax < 1 ? 1 : smax);
     int warps = (int)(SOLVE_SMEM_BUDGET / per_warp);
     if (warps < 1) return THANOS_ERR_SHAPE;
     if (warps > 8) warps = 8;
-    THANOS_CUDA(cudaFuncSetAttribute(solve_rows_general_kernel,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)SOLVE_SMEM_BUDGET));
+    {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_general_kernel, (int)SOLVE_SMEM_BUDGET, done));
+  }
     int64_t grid = ceil_div(c, warps);
     if (grid > 148 * 4) grid = 148 * 4;
     solve_rows_general_kernel<<<(unsigned)grid, warps * 32, per_warp * warps, stream>>>(
@@ -610,8 +612,11 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
   if (n_small + 1 <= 64)
     return launch_fast<2>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                           fixed_kind, rep, stats, stream);
-  return launch_fast<3>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc, fixed_kind,
-                        rep, stats, stream);
+  if (n_small + 1 <= 96)
+    return launch_fast<3>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
+                          fixed_kind, rep, stats, stream);
+  return launch_fast<5>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
+                        fixed_kind, rep, stats, stream);
 }
 
 }  // namespace thanos

@@ -479,8 +479,10 @@ thanos_status_t tc_gemm_split3(const TcGemmArgs& a, cudaStream_t stream) {
   if (tiles > (1ll << 30)) return THANOS_ERR_SHAPE;
   const int G = sm_count();
   const int grid = (int)(tiles < G ? tiles : G);
-  THANOS_CUDA(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)SMEM_BYTES));
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(tc_gemm_kernel, (int)SMEM_BYTES, done));
+  }
   tc_gemm_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(mapA, mapB, mapD, p);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
