@@ -55,54 +55,75 @@ __global__ void copy_damped_upper_kernel(const float* __restrict__ H, float* __r
 }
 
 // ---- diagonal block: A22 = V22 V22^T (V22 upper, i.e. Cholesky from the last row backwards) and
-//      U22 = inv(V22).  One CTA, one thread per row.  With the rows and columns reversed this is
-//      an ordinary lower Cholesky L; n identity rows appended below the block turn into L^{-T}
-//      under the same elimination, which gives the inverse without a second pass.
-//      Left-looking in panels of 8 columns; every thread factors the 8 x 8 diagonal piece itself.
-__global__ void __launch_bounds__(2 * NB)
+//      U22 = inv(V22).  One CTA.  With the rows and columns reversed this is an ordinary lower
+//      Cholesky L; n identity rows appended below the block turn into L^{-T} under the same
+//      elimination, which gives the inverse without a second pass.
+//      Left-looking in panels of 8 columns.  Two threads share a row and split the contraction
+//      range in alternating runs of 16 columns; every thread factors the 8 x 8 diagonal piece
+//      itself (reciprocal square roots by one Newton step on the hardware estimate).
+constexpr int DIAG_THREADS = 4 * NB;
+
+__global__ void __launch_bounds__(DIAG_THREADS)
 diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* __restrict__ Up,
                   int64_t plane, int b, int k0, int n, int32_t* __restrict__ status) {
   extern __shared__ __align__(16) float dsm[];
   float* L = dsm;                       // [2 n][DLD]
   float* dblk = dsm + 2 * NB * DLD;     // [8][8]
   const int tid = threadIdx.x;
-  for (int e = tid; e < n * n; e += blockDim.x) {
-    const int i = e / n, j = e - i * n;
-    float v = 0.f;
-    if (j <= i) v = V[(int64_t)(k0 + n - 1 - i) * b + k0 + n - 1 - j];
-    L[i * DLD + j] = v;
-    L[(n + i) * DLD + j] = (i == j) ? 1.f : 0.f;
+  const int warp = tid >> 5, lane = tid & 31;
+  // reversed lower triangle of the block, then the identity
+  for (int i = warp; i < n; i += DIAG_THREADS / 32) {
+    const float* src = V + (int64_t)(k0 + n - 1 - i) * b + k0;
+    for (int c4 = lane * 4; c4 < n; c4 += 128) {
+      const float4 v = *reinterpret_cast<const float4*>(src + c4);
+      const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = n - 1 - (c4 + u);
+        L[i * DLD + j] = (j <= i) ? e[u] : 0.f;
+        L[(n + i) * DLD + j] = (i == j) ? 1.f : 0.f;
+      }
+    }
   }
   __syncthreads();
-  const int r = tid;
+  const int r = tid >> 1;
+  const int half = tid & 1;
   const bool is_row = r < 2 * n;
   float* Lr = L + (is_row ? r : 0) * DLD;
-  // identity row j is zero left of column j: its products start there (rounded down per warp)
+  // identity row j is zero left of column j: its products start there (rounded down to 32)
   const int first_nz = (r >= n) ? ((r - n) & ~31) : 0;
   for (int c0 = 0; c0 < n; c0 += 8) {
     const bool active = is_row && r >= c0;
     float acc[8];
-    {
+    if (half == 0) {
       const float4 lo = *reinterpret_cast<const float4*>(Lr + c0);
       const float4 hi = *reinterpret_cast<const float4*>(Lr + c0 + 4);
       acc[0] = lo.x; acc[1] = lo.y; acc[2] = lo.z; acc[3] = lo.w;
       acc[4] = hi.x; acc[5] = hi.y; acc[6] = hi.z; acc[7] = hi.w;
+    } else {
+#pragma unroll
+      for (int w = 0; w < 8; ++w) acc[w] = 0.f;
     }
     if (active) {
       const float* Pb = L + c0 * DLD;
-      for (int k = first_nz; k < c0; k += 4) {
-        const float4 av = *reinterpret_cast<const float4*>(Lr + k);
+      for (int kk = first_nz + 16 * half; kk < c0; kk += 32) {
+        const int kend = kk + 16 < c0 ? kk + 16 : c0;
+        for (int k = kk; k < kend; k += 4) {
+          const float4 av = *reinterpret_cast<const float4*>(Lr + k);
 #pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          const float4 bv = *reinterpret_cast<const float4*>(Pb + w * DLD + k);
-          acc[w] = fmaf(-av.x, bv.x, acc[w]);
-          acc[w] = fmaf(-av.y, bv.y, acc[w]);
-          acc[w] = fmaf(-av.z, bv.z, acc[w]);
-          acc[w] = fmaf(-av.w, bv.w, acc[w]);
+          for (int w = 0; w < 8; ++w) {
+            const float4 bv = *reinterpret_cast<const float4*>(Pb + w * DLD + k);
+            acc[w] = fmaf(-av.x, bv.x, acc[w]);
+            acc[w] = fmaf(-av.y, bv.y, acc[w]);
+            acc[w] = fmaf(-av.z, bv.z, acc[w]);
+            acc[w] = fmaf(-av.w, bv.w, acc[w]);
+          }
         }
       }
     }
-    if (r >= c0 && r < c0 + 8) {
+#pragma unroll
+    for (int w = 0; w < 8; ++w) acc[w] += __shfl_xor_sync(0xffffffffu, acc[w], 1);
+    if (half == 0 && r >= c0 && r < c0 + 8) {
 #pragma unroll
       for (int w = 0; w < 8; ++w) dblk[(r - c0) * 8 + w] = acc[w];
     }
@@ -112,7 +133,7 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) ld[i][j] = dblk[i * 8 + j];
+      for (int j = 0; j <= i; ++j) ld[i][j] = dblk[i * 8 + j];
     float rinv[8];
 #pragma unroll
     for (int w = 0; w < 8; ++w) {
@@ -121,9 +142,11 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
         if (tid == 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + n - 1 - (c0 + w));
         d = 1.f;
       }
-      rinv[w] = 1.0f / sqrtf(d);
+      float ri = rsqrtf(d);
+      ri = ri * fmaf(-0.5f * d, ri * ri, 1.5f);
+      rinv[w] = ri;
 #pragma unroll
-      for (int v = w; v < 8; ++v) ld[v][w] *= rinv[w];
+      for (int v = w; v < 8; ++v) ld[v][w] *= ri;
 #pragma unroll
       for (int v = w + 1; v < 8; ++v)
 #pragma unroll
@@ -138,27 +161,41 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
       for (int v = 0; v < w; ++v) t = fmaf(-x[v], ld[w][v], t);
       x[w] = t * rinv[w];
     }
-    if (active) {
+    if (active && half == 0) {
       *reinterpret_cast<float4*>(Lr + c0) = make_float4(x[0], x[1], x[2], x[3]);
       *reinterpret_cast<float4*>(Lr + c0 + 4) = make_float4(x[4], x[5], x[6], x[7]);
     }
     __syncthreads();
   }
   // V22[i][j] = L[n-1-i][n-1-j];  U22[i][j] = inv(L)[n-1-i][n-1-j] = extra row (n-1-j), column n-1-i
-  for (int e = tid; e < n * n; e += blockDim.x) {
-    const int i = e / n, j = e - i * n;
-    float u = 0.f;
-    if (j >= i) {
-      V[(int64_t)(k0 + i) * b + k0 + j] = L[(n - 1 - i) * DLD + (n - 1 - j)];
-      u = L[(n + n - 1 - j) * DLD + (n - 1 - i)];
-    }
-    const int64_t o = (int64_t)(k0 + i) * b + k0 + j;
-    U[o] = u;
+  for (int i = warp; i < n; i += DIAG_THREADS / 32) {
+    for (int c4 = lane * 4; c4 < n; c4 += 128) {
+      float u4[4];
+      const int64_t o = (int64_t)(k0 + i) * b + k0 + c4;
 #pragma unroll
-    for (int pl = 0; pl < 3; ++pl) {
-      const __nv_bfloat16 hb = __float2bfloat16_rn(u);
-      Up[(int64_t)pl * plane + o] = hb;
-      u -= __bfloat162float(hb);
+      for (int e = 0; e < 4; ++e) {
+        const int j = c4 + e;
+        float u = 0.f;
+        if (j >= i) {
+          V[o + e] = L[(n - 1 - i) * DLD + (n - 1 - j)];
+          u = L[(n + n - 1 - j) * DLD + (n - 1 - i)];
+        }
+        u4[e] = u;
+      }
+      *reinterpret_cast<float4*>(U + o) = make_float4(u4[0], u4[1], u4[2], u4[3]);
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl) {
+        __nv_bfloat16 hb[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          hb[e] = __float2bfloat16_rn(u4[e]);
+          u4[e] -= __bfloat162float(hb[e]);
+        }
+        uint2 pk;
+        pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) | ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
+        pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) | ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
+        *reinterpret_cast<uint2*>(Up + (int64_t)pl * plane + o) = pk;
+      }
     }
   }
 }
@@ -227,7 +264,7 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
   for (int kb = nblk - 1; kb >= 0; --kb) {
     const int k0 = kb * NB;
     const int n = (b - k0 < NB) ? b - k0 : NB;
-    diag_block_kernel<<<1, 2 * NB, DIAG_SMEM, stream>>>(w.V, factor, w.Up, plane, b, k0, n,
+    diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(w.V, factor, w.Up, plane, b, k0, n,
                                                        status_dev);
     THANOS_CHECK_LAUNCH();
     if (k0 == 0) break;
@@ -276,43 +313,60 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
   //      U12 = -U11 (V12 U22)
   for (int64_t sz = NB; sz < b; sz *= 2) {
     const int npairs = (int)ceil_div(b, 2 * sz);
-    for (int t = 0; t < npairs; ++t) {
+    // pairs whose second block is a full sz wide go out as one batched product per step; a
+    // ragged last pair follows on its own
+    int nfull = 0;
+    while (nfull < npairs && (int64_t)(2 * nfull + 2) * sz <= b) ++nfull;
+    for (int part = 0; part < 2; ++part) {
+      const int t = part == 0 ? 0 : nfull;
+      const int cnt = part == 0 ? nfull : npairs - nfull;
+      if (cnt <= 0) continue;
       const int64_t r0 = 2 * t * sz, c0 = r0 + sz;
-      if (c0 >= b) break;
+      if (c0 >= b) continue;
       const int N = (int)((c0 + sz < b ? c0 + sz : b) - c0);
+      const int64_t pair_stride = 2 * sz * ((int64_t)b + 1);
       __nv_bfloat16* Tt = w.Tp + (size_t)t * sz * sz;
       TcGemmArgs g;
       g.Dp = Tt;
       g.ldp = N;
       g.dp_plane = (int64_t)w.t_elems;
+      g.dp_batch = sz * sz;
       g.A = w.Vp + r0 * b + c0;
       g.lda = b;
       g.a_plane = plane;
+      g.a_batch = pair_stride;
       g.B = w.Up + c0 * b + c0;
       g.ldb = b;
       g.b_plane = plane;
+      g.b_batch = pair_stride;
       g.b_kmajor = 0;
       g.M = (int)sz;
       g.N = N;
       g.K = N;
+      g.batch = part == 0 ? cnt : 1;
       g.status = w.tc_status;
       THANOS_TRY(tc_gemm_split3(g, stream));
       TcGemmArgs h;
       h.D = factor + r0 * b + c0;
       h.ldd = b;
+      h.d_batch = pair_stride;
       h.Dp = w.Up + r0 * b + c0;
       h.ldp = b;
       h.dp_plane = plane;
+      h.dp_batch = pair_stride;
       h.A = w.Up + r0 * b + r0;
       h.lda = b;
       h.a_plane = plane;
+      h.a_batch = pair_stride;
       h.B = Tt;
       h.ldb = N;
       h.b_plane = (int64_t)w.t_elems;
+      h.b_batch = sz * sz;
       h.b_kmajor = 0;
       h.M = (int)sz;
       h.N = N;
       h.K = (int)sz;
+      h.batch = part == 0 ? cnt : 1;
       h.alpha = -1.f;
       h.status = w.tc_status;
       THANOS_TRY(tc_gemm_split3(h, stream));
