@@ -26,21 +26,43 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
 
 namespace {
 
-// Radix select over the 31 significant key bits (metric >= 0): four passes of 8, 8, 8, 7 bits.
-constexpr int NPASS = 4;
-constexpr int HIST_BINS = 256;
+// Selection of the block threshold: the r-th smallest metric key over the residual (Eq. psi with
+// the running budget r of Algorithm 1).  Keys are the fp32 bit patterns of |w| * ||X_j|| (>= 0, so
+// they order like the values).  Two routes, both exact:
+//   bracket  the threshold moves little from block to block, so one pass counts the keys below a
+//            window of 2^18 key values around the previous threshold and bins the keys inside it
+//            (512 bins of 512 values); a second pass resolves the 512 values of the hit bin;
+//   radix    four passes over 8, 8, 8 and 7 key bits (first block, or when the window misses).
+// One kernel, launched five times per block, does whichever pass the sweep state asks for; the
+// last CTA to finish a pass reads the histogram, decides and sets the next phase.
+constexpr int HIST_BINS = 512;
+constexpr int RADIX_BINS = 256;
+constexpr unsigned WINDOW = 1u << 18;   // key values covered by the bracket
+constexpr int WINDOW_SHIFT = 9;         // 512 values per bracket bin
 __host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0)); }
 
+enum SelectPhase : int {
+  PH_RADIX0 = 0, PH_RADIX1 = 1, PH_RADIX2 = 2, PH_RADIX3 = 3, PH_BRACKET = 4, PH_REFINE = 5,
+  PH_DONE = 6
+};
+
 struct SweepState {
   long long r;                   // removals still to place before the current block
-  unsigned long long k_rem;      // rank still to resolve inside the current candidate bin
+  unsigned long long k_rem;      // rank still to resolve inside the current candidate range
   unsigned long long need_eq;    // how many entries with key == tau are removed
   unsigned long long count_eq;   // how many entries with key == tau the residual holds
   unsigned long long blk_count;  // entries removed in the current block
-  unsigned int prefix;           // key bits fixed so far
+  unsigned long long below;      // bracket pass: keys below the window
+  unsigned int prefix;           // radix: key bits fixed so far
   unsigned int tau;              // threshold key of the current block
+  unsigned int lo;               // start of the bracket window / of the bin being refined
+  unsigned int tau_prev;         // threshold of the previous block
+  int have_prev;
   int none;                      // nothing to remove in this block
+  int phase;                     // what the next select pass does
+  unsigned int ticket;           // CTAs that have finished the current pass
+  unsigned int mark_ticket;      // same for the mask kernel
   int pad;
 };
 
@@ -149,100 +171,204 @@ block_rows_kernel(const float* __restrict__ U, const float* __restrict__ Vbb,
 }
 
 // ------------------------------------------------------------------ unstructured selection
-__global__ void begin_block_kernel(SweepState* st, const int64_t* r_ext, unsigned* list_counts) {
-  list_counts[0] = list_counts[1] = 0;
-  if (r_ext) st->r = *r_ext;
-  st->none = (st->r <= 0) ? 1 : 0;
-  st->k_rem = st->r > 0 ? (unsigned long long)st->r : 0ull;
-  st->prefix = 0;
-  st->blk_count = 0;
-  st->need_eq = 0;
-  st->count_eq = 0;
-}
-
-// Histogram of one radix digit over the residual.  The shared histogram keeps one counter per
-// (bin, lane): a warp never hits the same bank twice, whatever the skew of the metric.
-template <int PASS>
-__global__ void __launch_bounds__(256)
-hist_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
-                 int j1, const SweepState* __restrict__ st, unsigned* __restrict__ hist) {
-  constexpr int BITS = pass_bits(PASS);
-  constexpr int SHIFT = pass_shift(PASS);
-  constexpr int NBIN = 1 << BITS;
-  __shared__ unsigned sh[NBIN * 32];
-  if (st->none) return;
-  for (int i = threadIdx.x; i < NBIN * 32; i += 256) sh[i] = 0;
-  __syncthreads();
-  const unsigned prefix = st->prefix;
+// Warp scan over NBIN (<= 512) histogram bins: finds the bin that holds rank k (1-based) and
+// returns (bin, entries before it, entries in it) to every lane; bin = -1 if k is out of range.
+__device__ __forceinline__ void find_rank_bin(const unsigned* hist, int nbin, unsigned long long k,
+                                              int& bin_out, unsigned long long& before_out,
+                                              unsigned long long& inbin_out) {
   const int lane = threadIdx.x & 31;
-  const int w4 = (b - j1) >> 2;
-  const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
-  for (int row = blockIdx.x; row < c; row += gridDim.x) {
-    const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-    for (int q = threadIdx.x; q < w4; q += 256) {
-      float4 w = wr[q];
-      float4 x = __ldg(&xr[q]);
-      unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
-                       metric_key(w.w, x.w)};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (PASS == 0 || (k[e] >> (SHIFT + BITS)) == prefix)
-          atomicAdd(&sh[((k[e] >> SHIFT) & (NBIN - 1)) * 32 + lane], 1u);
-      }
-    }
-  }
-  __syncthreads();
-  for (int bin = threadIdx.x; bin < NBIN; bin += 256) {
-    unsigned t = 0;
-#pragma unroll
-    for (int l = 0; l < 32; ++l) t += sh[bin * 32 + ((l + bin) & 31)];
-    if (t) atomicAdd(&hist[bin], t);
-  }
-}
-
-// One warp: locate the bin holding the k_rem-th smallest candidate, extend the prefix.
-template <int PASS>
-__global__ void __launch_bounds__(32)
-scan_pass_kernel(SweepState* st, unsigned* __restrict__ hist) {
-  constexpr int BITS = pass_bits(PASS);
-  constexpr int NBIN = 1 << BITS;
   constexpr int PER = HIST_BINS / 32;
-  if (st->none) return;
-  const int lane = threadIdx.x;
   unsigned long long loc[PER];
   unsigned long long tsum = 0;
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
-    int bin = lane * PER + e;
-    loc[e] = bin < NBIN ? hist[bin] : 0;
+    const int bin = lane * PER + e;
+    loc[e] = bin < nbin ? (unsigned long long)__ldcg(&hist[bin]) : 0ull;
     tsum += loc[e];
   }
   unsigned long long inc = tsum;
   for (int o = 1; o < 32; o <<= 1) {
-    unsigned long long v = __shfl_up_sync(0xffffffffu, inc, o);
+    const unsigned long long v = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += v;
   }
-  const unsigned long long k = st->k_rem;
-  const unsigned prefix = st->prefix;
-  __syncwarp();
   unsigned long long excl = inc - tsum;
+  int found = -1;
+  unsigned long long fb = 0, fi = 0;
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
-    int bin = lane * PER + e;
-    if (bin < NBIN && excl < k && k <= excl + loc[e]) {
-      const unsigned np = (prefix << BITS) | (unsigned)bin;
-      st->prefix = np;
-      st->k_rem = k - excl;
-      if (PASS == NPASS - 1) {
-        st->tau = np;
-        st->need_eq = k - excl;
-        st->count_eq = loc[e];
-      }
+    if (found < 0 && k > excl && k <= excl + loc[e]) {
+      found = lane * PER + e;
+      fb = excl;
+      fi = loc[e];
     }
     excl += loc[e];
   }
+  const unsigned has = __ballot_sync(0xffffffffu, found >= 0);
+  if (has == 0) {
+    bin_out = -1;
+    before_out = inbin_out = 0;
+    return;
+  }
+  const int src = __ffs(has) - 1;
+  bin_out = __shfl_sync(0xffffffffu, found, src);
+  before_out = __shfl_sync(0xffffffffu, fb, src);
+  inbin_out = __shfl_sync(0xffffffffu, fi, src);
+}
+
+// One pass of the threshold selection over the residual W[:, j1:]; what it does is st->phase.
+// Shared histogram: radix passes keep one counter per (bin, lane) -- a warp never hits the same
+// bank twice, whatever the skew of the metric; bracket / refine passes see few keys inside
+// their range and use plain counters.
+__global__ void __launch_bounds__(256)
+select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
+                   int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
+                   unsigned* __restrict__ list_counts, int first_launch) {
+  __shared__ unsigned sh[RADIX_BINS * 32];
+  __shared__ int s_last;
+  const int phase = st->phase;
+  if (phase == PH_DONE && !first_launch) return;
+  if (first_launch && blockIdx.x == 0 && threadIdx.x == 0) {
+    list_counts[0] = list_counts[1] = 0;
+    if (r_ext) st->r = *r_ext;
+  }
+  const int lane = threadIdx.x & 31;
+  const int w4 = (b - j1) >> 2;
+  const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
+  const bool radix = phase <= PH_RADIX3;
+  const int nclear = radix ? RADIX_BINS * 32 : HIST_BINS;
+  for (int i = threadIdx.x; i < nclear; i += 256) sh[i] = 0;
+  __syncthreads();
+  unsigned below = 0;
+  if (radix) {
+    const int shift = pass_shift(phase), bits = pass_bits(phase);
+    const unsigned prefix = st->prefix;
+    const unsigned bmask = (1u << bits) - 1u;
+    for (int row = blockIdx.x; row < c; row += gridDim.x) {
+      const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+      for (int q = threadIdx.x; q < w4; q += 256) {
+        const float4 w = wr[q];
+        const float4 x = __ldg(&xr[q]);
+        const unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
+                               metric_key(w.w, x.w)};
 #pragma unroll
-  for (int e = 0; e < PER; ++e) hist[lane * PER + e] = 0;
+        for (int e = 0; e < 4; ++e) {
+          if (phase == PH_RADIX0 || (k[e] >> (shift + bits)) == prefix)
+            atomicAdd(&sh[((k[e] >> shift) & bmask) * 32 + lane], 1u);
+        }
+      }
+    }
+  } else {
+    const unsigned lo = st->lo;
+    const unsigned width = phase == PH_BRACKET ? WINDOW : (unsigned)HIST_BINS;
+    const int bshift = phase == PH_BRACKET ? WINDOW_SHIFT : 0;
+    for (int row = blockIdx.x; row < c; row += gridDim.x) {
+      const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+      for (int q = threadIdx.x; q < w4; q += 256) {
+        const float4 w = wr[q];
+        const float4 x = __ldg(&xr[q]);
+        const unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
+                               metric_key(w.w, x.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned d = k[e] - lo;
+          if (k[e] < lo) ++below;
+          else if (d < width) atomicAdd(&sh[d >> bshift], 1u);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (radix) {
+    const int nbin = 1 << pass_bits(phase);
+    for (int bin = threadIdx.x; bin < nbin; bin += 256) {
+      unsigned t = 0;
+#pragma unroll
+      for (int l = 0; l < 32; ++l) t += sh[bin * 32 + ((l + bin) & 31)];
+      if (t) atomicAdd(&hist[bin], t);
+    }
+  } else {
+    for (int bin = threadIdx.x; bin < HIST_BINS; bin += 256)
+      if (sh[bin]) atomicAdd(&hist[bin], sh[bin]);
+    if (phase == PH_BRACKET) {
+      for (int o = 16; o > 0; o >>= 1) below += __shfl_down_sync(0xffffffffu, below, o);
+      if (lane == 0 && below) atomicAdd(&st->below, (unsigned long long)below);
+    }
+  }
+  // ---- the last CTA to get here decides
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(&st->ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+  __syncthreads();
+  if (!s_last || threadIdx.x >= 32) return;
+  __threadfence();
+  volatile SweepState* vs = st;
+  const unsigned* vh = hist;
+  int next = PH_DONE;
+  if (first_launch) {
+    const long long r = vs->r;
+    if (lane == 0) {
+      st->none = r <= 0 ? 1 : 0;
+      st->k_rem = r > 0 ? (unsigned long long)r : 0ull;
+      st->blk_count = 0;
+      st->need_eq = 0;
+      st->count_eq = 0;
+    }
+    __syncwarp();
+  }
+  const bool none = vs->none != 0;
+  const unsigned long long k = vs->k_rem;
+  if (none) {
+    next = PH_DONE;
+  } else if (radix) {
+    int bin;
+    unsigned long long before, inbin;
+    find_rank_bin(const_cast<const unsigned*>(vh), 1 << pass_bits(phase), k, bin, before, inbin);
+    if (bin < 0) bin = 0;  // cannot happen: k <= number of candidates
+    const unsigned np = (vs->prefix << pass_bits(phase)) | (unsigned)bin;
+    if (lane == 0) {
+      st->prefix = phase == PH_RADIX3 ? 0u : np;
+      st->k_rem = k - before;
+      if (phase == PH_RADIX3) {
+        st->tau = np;
+        st->need_eq = k - before;
+        st->count_eq = inbin;
+      }
+    }
+    next = phase == PH_RADIX3 ? PH_DONE : phase + 1;
+  } else if (phase == PH_BRACKET) {
+    const unsigned long long bel = vs->below;
+    int bin = -1;
+    unsigned long long before = 0, inbin = 0;
+    if (k > bel) find_rank_bin(const_cast<const unsigned*>(vh), HIST_BINS, k - bel, bin, before, inbin);
+    if (bin >= 0) {
+      if (lane == 0) {
+        st->lo = vs->lo + ((unsigned)bin << WINDOW_SHIFT);
+        st->k_rem = k - bel - before;
+      }
+      next = PH_REFINE;
+    } else {
+      if (lane == 0) st->prefix = 0;
+      next = PH_RADIX0;  // the window missed: full radix select, k_rem is still the rank
+    }
+  } else {  // PH_REFINE
+    int bin;
+    unsigned long long before, inbin;
+    find_rank_bin(const_cast<const unsigned*>(vh), HIST_BINS, k, bin, before, inbin);
+    if (bin < 0) bin = 0;  // cannot happen: the bracket pass counted this bin
+    if (lane == 0) {
+      st->tau = vs->lo + (unsigned)bin;
+      st->need_eq = k - before;
+      st->count_eq = inbin;
+    }
+    next = PH_DONE;
+  }
+  __syncwarp();
+  for (int i = lane; i < HIST_BINS; i += 32) hist[i] = 0;
+  if (lane == 0) {
+    st->below = 0;
+    st->ticket = 0;
+    st->phase = next;
+  }
 }
 
 // Rows' counts of entries equal to the threshold over the residual (only needed when the
@@ -317,7 +443,8 @@ __global__ void __launch_bounds__(256)
 mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
                   uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, SweepState* st,
                   const unsigned long long* __restrict__ rowbase, int* __restrict__ row_lists,
-                  unsigned* __restrict__ list_counts, thanos_stats_t* stats) {
+                  unsigned* __restrict__ list_counts, thanos_stats_t* stats, int64_t* r_ext) {
+  __shared__ int s_last;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const bool none = st->none != 0;
@@ -358,14 +485,47 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
     if (total) atomicAdd(&st->blk_count, total);
     if (smax) atomicMax(&stats->max_s, smax);
   }
+  // ---- the last CTA closes the block: budget, statistics, state of the next block's selection
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(&st->mark_ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+  __syncthreads();
+  if (!s_last || threadIdx.x != 0) return;
+  __threadfence();
+  volatile SweepState* vs = st;
+  const unsigned long long cnt = vs->blk_count;
+  const long long r_new = vs->r - (long long)cnt;
+  st->r = r_new;
+  stats->r_left = r_new;
+  if (!none) {
+    stats->n_tied += (long long)(vs->count_eq - vs->need_eq);
+    stats->last_threshold_bits = tau;
+    st->tau_prev = tau;
+  }
+  if (r_ext) *r_ext = r_new;
+  stats->n_pruned += (long long)cnt;
+  stats->n_blocks += 1;
+  st->blk_count = 0;
+  st->mark_ticket = 0;
+  // next block: bracket around this threshold when there is one, else a full radix select
+  const bool bracket = !none && tau >= (WINDOW >> 1);
+  st->have_prev = bracket ? 1 : 0;
+  st->lo = bracket ? tau - (WINDOW >> 1) : 0u;
+  st->prefix = 0;
+  st->phase = bracket ? PH_BRACKET : PH_RADIX0;
 }
 
 // n:m: one thread per (row, group of m columns); the n smallest keys, lower column on ties.
 __global__ void __launch_bounds__(256)
 nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
-               uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, int n, int m) {
+               uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, int n, int m,
+               thanos_stats_t* stats) {
   const int groups = Bw / m;
   int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx == 0) {  // launches of one sweep are ordered, so one thread can keep the books
+    stats->n_pruned += (long long)c * groups * n;
+    stats->n_blocks += 1;
+  }
   if (idx >= (int64_t)c * groups) return;
   int row = (int)(idx / groups), g = (int)(idx % groups);
   const float* w = Wc + (int64_t)row * b + j1 + g * m;
@@ -381,22 +541,8 @@ nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
   }
 }
 
-__global__ void finish_block_kernel(SweepState* st, thanos_stats_t* stats, int64_t* r_ext,
-                                    long long nm_count, int is_nm, const int32_t* tc_status) {
+__global__ void fold_tc_status_kernel(thanos_stats_t* stats, const int32_t* tc_status) {
   if (*tc_status != 0 && stats->status == 0) stats->status = *tc_status;
-  unsigned long long cnt = is_nm ? (unsigned long long)nm_count : st->blk_count;
-  if (!is_nm) {
-    st->r -= (long long)cnt;
-    stats->r_left = st->r;
-    if (!st->none) {
-      stats->n_tied += (long long)(st->count_eq - st->need_eq);
-      stats->last_threshold_bits = st->tau;
-    }
-    if (r_ext) *r_ext = st->r;
-  }
-  stats->n_pruned += (long long)cnt;
-  stats->n_blocks += 1;
-  st->blk_count = 0;
 }
 
 // ------------------------------------------------------------------ dtype conversion
@@ -415,11 +561,10 @@ __global__ void to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __re
 }
 
 __global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long long r) {
-  st->r = r;
-  st->k_rem = 0;
-  st->need_eq = st->count_eq = st->blk_count = 0;
-  st->prefix = st->tau = 0;
-  st->none = 0;
+  SweepState z0 = {};
+  z0.r = r;
+  z0.phase = PH_RADIX0;
+  *st = z0;
   thanos_stats_t z = {};
   z.r_left = r;
   *stats = z;
@@ -491,24 +636,12 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
     int hg = c < 148 * 8 ? c : 148 * 8;
-    begin_block_kernel<<<1, 1, 0, stream>>>(w.st, r_ext, w.list_counts);
-    THANOS_CHECK_LAUNCH();
-    hist_pass_kernel<0><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<0><<<1, 32, 0, stream>>>(w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    hist_pass_kernel<1><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<1><<<1, 32, 0, stream>>>(w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    hist_pass_kernel<2><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<2><<<1, 32, 0, stream>>>(w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    hist_pass_kernel<3><<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
-    scan_pass_kernel<3><<<1, 32, 0, stream>>>(w.st, w.hist);
-    THANOS_CHECK_LAUNCH();
+    // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
+    for (int pass = 0; pass < 5; ++pass) {
+      select_pass_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                 w.list_counts, pass == 0 ? 1 : 0);
+      THANOS_CHECK_LAUNCH();
+    }
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
     THANOS_CHECK_LAUNCH();
     tie_scan_kernel<<<1, 1024, 0, stream>>>(c, w.st, w.rowcnt, w.rowbase);
@@ -516,13 +649,13 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     int mg = (int)ceil_div(c, 8);
     if (mg > 148 * 8) mg = 148 * 8;
     mark_block_kernel<<<mg, 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
-                                              w.row_lists, w.list_counts, stats);
+                                              w.row_lists, w.list_counts, stats, r_ext);
     THANOS_CHECK_LAUNCH();
   } else {
     s_fixed = Bw / m * n;
     int64_t items = (int64_t)c * (Bw / m);
     nm_mark_kernel<<<(unsigned)ceil_div(items, 256), 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1,
-                                                                      Bw, n, m);
+                                                                      Bw, n, m, stats);
     THANOS_CHECK_LAUNCH();
   }
   THANOS_TRY(launch_block_solve(Wc, mask, w.G + (size_t)bb * B * B, w.S + (size_t)bb * B * B, B,
@@ -548,10 +681,6 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     g.status = w.tc_status;
     THANOS_TRY(tc_gemm_split3(g, stream));
   }
-  long long nm_count = mode == THANOS_NM ? (long long)c * (Bw / m) * n : 0;
-  finish_block_kernel<<<1, 1, 0, stream>>>(w.st, stats, r_ext, nm_count, mode == THANOS_NM,
-                                           w.tc_status);
-  THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
 
@@ -601,8 +730,11 @@ thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b,
   THANOS_CUDA(cudaMemsetAsync(w.st, 0, sizeof(SweepState), stream));
   THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
-  return block_step(Wc, mask, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
-                    stream);
+  THANOS_TRY(block_step(Wc, mask, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
+                        stream));
+  fold_tc_status_kernel<<<1, 1, 0, stream>>>(stats, w.tc_status);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
 }
 
 thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
@@ -636,6 +768,8 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
     THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr, w,
                           stats, stream));
   }
+  fold_tc_status_kernel<<<1, 1, 0, stream>>>(stats, w.tc_status);
+  THANOS_CHECK_LAUNCH();
   if (need_wc) {
     to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(Wc, static_cast<__nv_bfloat16*>(W_out), nel);
     THANOS_CHECK_LAUNCH();
