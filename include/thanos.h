@@ -69,7 +69,9 @@ typedef struct {
   int64_t n_tied;       /* unstructured: entries whose metric equals a block threshold
                            bit-for-bit but which the (row, column) tie-break left unpruned */
   uint32_t last_threshold_bits; /* fp32 bit pattern of the last block's threshold metric  */
-  int32_t reserved[5];
+  int32_t select_misses; /* unstructured: blocks whose threshold fell outside the bracket around
+                            the previous block's (they take the four-pass route)              */
+  int32_t reserved[4];
 } thanos_stats_t;
 
 /*

@@ -32,7 +32,8 @@ class _Stats(ctypes.Structure):
         ("n_blocks", ctypes.c_int32),
         ("n_tied", ctypes.c_int64),
         ("last_threshold_bits", ctypes.c_uint32),
-        ("reserved", ctypes.c_int32 * 5),
+        ("select_misses", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 4),
     ]
 
 
@@ -49,12 +50,13 @@ class PruneStats:
     n_blocks: int
     n_tied: int
     last_threshold_bits: int
+    select_misses: int = 0
 
     @staticmethod
     def from_bytes(raw: bytes) -> "PruneStats":
         s = _Stats.from_buffer_copy(raw)
         return PruneStats(s.status, s.err_index, s.n_pruned, s.r_left, s.max_s, s.n_blocks,
-                          s.n_tied, s.last_threshold_bits)
+                          s.n_tied, s.last_threshold_bits, s.select_misses)
 
 
 _lib = None

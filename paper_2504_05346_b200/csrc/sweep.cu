@@ -37,6 +37,7 @@ namespace {
 // last CTA to finish a pass reads the histogram, decides and sets the next phase.
 constexpr int HIST_BINS = 512;
 constexpr int RADIX_BINS = 256;
+constexpr int RADIX_REPL = 8;           // shared-memory copies of a radix histogram (by lane & 7)
 constexpr unsigned WINDOW = 1u << 18;   // key values covered by the bracket
 constexpr int WINDOW_SHIFT = 9;         // 512 values per bracket bin
 __host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
@@ -222,9 +223,10 @@ __device__ __forceinline__ void find_rank_bin(const unsigned* hist, int nbin, un
 __global__ void __launch_bounds__(256)
 select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                    int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
-                   unsigned* __restrict__ list_counts, int first_launch) {
-  __shared__ unsigned sh[RADIX_BINS * 32];
+                   unsigned* __restrict__ list_counts, int first_launch, thanos_stats_t* stats) {
+  __shared__ unsigned sh[RADIX_BINS * RADIX_REPL];
   __shared__ int s_last;
+  __shared__ unsigned s_below;
   const int phase = st->phase;
   if (phase == PH_DONE && !first_launch) return;
   if (first_launch && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -235,8 +237,9 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
   const int w4 = (b - j1) >> 2;
   const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
   const bool radix = phase <= PH_RADIX3;
-  const int nclear = radix ? RADIX_BINS * 32 : HIST_BINS;
+  const int nclear = radix ? RADIX_BINS * RADIX_REPL : HIST_BINS;
   for (int i = threadIdx.x; i < nclear; i += 256) sh[i] = 0;
+  if (threadIdx.x == 0) s_below = 0;
   __syncthreads();
   unsigned below = 0;
   if (radix) {
@@ -245,15 +248,24 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     const unsigned bmask = (1u << bits) - 1u;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-      for (int q = threadIdx.x; q < w4; q += 256) {
-        const float4 w = wr[q];
-        const float4 x = __ldg(&xr[q]);
-        const unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
-                               metric_key(w.w, x.w)};
+      for (int q0 = threadIdx.x; q0 < w4; q0 += 4 * 256) {
+        float4 w[4], x[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (phase == PH_RADIX0 || (k[e] >> (shift + bits)) == prefix)
-            atomicAdd(&sh[((k[e] >> shift) & bmask) * 32 + lane], 1u);
+        for (int u = 0; u < 4; ++u) {  // four loads in flight per thread
+          const int q = q0 + u * 256;
+          w[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[u] = q < w4 ? __ldg(&xr[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (q0 + u * 256 >= w4) break;
+          const unsigned k[4] = {metric_key(w[u].x, x[u].x), metric_key(w[u].y, x[u].y),
+                                 metric_key(w[u].z, x[u].z), metric_key(w[u].w, x[u].w)};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (phase == PH_RADIX0 || (k[e] >> (shift + bits)) == prefix)
+              atomicAdd(&sh[((k[e] >> shift) & bmask) * RADIX_REPL + (lane & (RADIX_REPL - 1))], 1u);
+          }
         }
       }
     }
@@ -263,16 +275,25 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     const int bshift = phase == PH_BRACKET ? WINDOW_SHIFT : 0;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-      for (int q = threadIdx.x; q < w4; q += 256) {
-        const float4 w = wr[q];
-        const float4 x = __ldg(&xr[q]);
-        const unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
-                               metric_key(w.w, x.w)};
+      for (int q0 = threadIdx.x; q0 < w4; q0 += 4 * 256) {
+        float4 w[4], x[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const unsigned d = k[e] - lo;
-          if (k[e] < lo) ++below;
-          else if (d < width) atomicAdd(&sh[d >> bshift], 1u);
+        for (int u = 0; u < 4; ++u) {  // four loads in flight per thread
+          const int q = q0 + u * 256;
+          w[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[u] = q < w4 ? __ldg(&xr[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (q0 + u * 256 >= w4) break;
+          const unsigned k[4] = {metric_key(w[u].x, x[u].x), metric_key(w[u].y, x[u].y),
+                                 metric_key(w[u].z, x[u].z), metric_key(w[u].w, x[u].w)};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const unsigned d = k[e] - lo;
+            if (k[e] < lo) ++below;
+            else if (d < width) atomicAdd(&sh[d >> bshift], 1u);
+          }
         }
       }
     }
@@ -283,7 +304,7 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     for (int bin = threadIdx.x; bin < nbin; bin += 256) {
       unsigned t = 0;
 #pragma unroll
-      for (int l = 0; l < 32; ++l) t += sh[bin * 32 + ((l + bin) & 31)];
+      for (int l = 0; l < RADIX_REPL; ++l) t += sh[bin * RADIX_REPL + l];
       if (t) atomicAdd(&hist[bin], t);
     }
   } else {
@@ -291,7 +312,9 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       if (sh[bin]) atomicAdd(&hist[bin], sh[bin]);
     if (phase == PH_BRACKET) {
       for (int o = 16; o > 0; o >>= 1) below += __shfl_down_sync(0xffffffffu, below, o);
-      if (lane == 0 && below) atomicAdd(&st->below, (unsigned long long)below);
+      if (lane == 0 && below) atomicAdd(&s_below, below);
+      __syncthreads();
+      if (threadIdx.x == 0 && s_below) atomicAdd(&st->below, (unsigned long long)s_below);
     }
   }
   // ---- the last CTA to get here decides
@@ -347,7 +370,10 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       }
       next = PH_REFINE;
     } else {
-      if (lane == 0) st->prefix = 0;
+      if (lane == 0) {
+        st->prefix = 0;
+        stats->select_misses += 1;
+      }
       next = PH_RADIX0;  // the window missed: full radix select, k_rem is still the rank
     }
   } else {  // PH_REFINE
@@ -637,9 +663,10 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (mode == THANOS_UNSTRUCTURED) {
     int hg = c < 148 * 8 ? c : 148 * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
+    const int sg = c < 148 * 4 ? c : 148 * 4;
     for (int pass = 0; pass < 5; ++pass) {
-      select_pass_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
-                                                 w.list_counts, pass == 0 ? 1 : 0);
+      select_pass_kernel<<<sg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                 w.list_counts, pass == 0 ? 1 : 0, stats);
       THANOS_CHECK_LAUNCH();
     }
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
