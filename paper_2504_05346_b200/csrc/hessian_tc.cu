@@ -394,6 +394,10 @@ constexpr int SPLIT_CHUNK = 8192;  // tokens of fp32 input split per pass
 
 }  // namespace
 
+bool hessian_tc2_supported(int64_t b, int64_t n_tok);
+thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, int64_t ld_elems,
+                                   int n_tok, int32_t* status, cudaStream_t stream);
+
 size_t hessian_tc_workspace_bytes(int64_t b, thanos_dtype_t dtype) {
   size_t w = 256;  // status word
   if (dtype == THANOS_F32) w += round_up((size_t)3 * SPLIT_CHUNK * b * sizeof(__nv_bfloat16), 256);
@@ -412,6 +416,12 @@ thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos
     const int64_t step = (int64_t)1 << 22;
     for (int64_t t0 = 0; t0 < n_tok; t0 += step) {
       int64_t n = n_tok - t0 < step ? n_tok - t0 : step;
+      if (hessian_tc2_supported(b, n)) {  // CTA pairs; falls through if they cannot be scheduled
+        thanos_status_t st2 = launch_hessian_tc2(
+            H, (int)b, static_cast<const __nv_bfloat16*>(X) + t0 * ldx, ldx, (int)n, status, stream);
+        if (st2 == THANOS_OK) continue;
+        if (st2 != THANOS_ERR_SHAPE) return st2;
+      }
       THANOS_TRY(launch_tc(H, (int)b, static_cast<const __nv_bfloat16*>(X) + t0 * ldx, ldx, (int)n,
                            1, n * ldx, status, stream));
     }
