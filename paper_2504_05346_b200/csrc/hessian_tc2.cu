@@ -398,20 +398,21 @@ thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, i
   const int nT = (b + TT - 1) / TT;
   p.n_tiles = nT * (nT + 1) / 2;
   // token slices: the count (each slice >= 2048 tokens) that wastes the least of the last wave
-  int best_s = 1;
-  double best_eff = 0.0;
+  // fewest slices whose last wave wastes at most 3 percent more than the best count does:
+  // longer slices mean fewer write-outs of a tile
   int max_s = n_tok / 2048;
   if (max_s < 1) max_s = 1;
   if (max_s > 16) max_s = 16;
+  double eff_of[17];
+  double best_eff = 0.0;
   for (int s = 1; s <= max_s; ++s) {
     const long long units = (long long)p.n_tiles * s;
     const long long waves = (units + G - 1) / G;
-    const double eff = (double)units / (double)(waves * G);
-    if (eff > best_eff + 1e-9) {
-      best_eff = eff;
-      best_s = s;
-    }
+    eff_of[s] = (double)units / (double)(waves * G);
+    if (eff_of[s] > best_eff) best_eff = eff_of[s];
   }
+  int best_s = 1;
+  while (best_s < max_s && eff_of[best_s] < best_eff - 0.03) ++best_s;
   int st = (n_tok + best_s - 1) / best_s;
   st = (st + FLUSH_STAGES * BK - 1) / (FLUSH_STAGES * BK) * (FLUSH_STAGES * BK);
   p.slice_tokens = st;
