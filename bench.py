@@ -91,6 +91,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """The slowest rank's time: one all_reduce(MAX) over the default process group (any backend);
+    the value itself when no group is up.  Replicas exchange nothing else."""
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(weights_per_replica: int, steps: int, world: int, ms_total: float) -> float:
+    """Weights swept per second by all replicas together, given the slowest rank's time."""
+    return world * weights_per_replica * steps / (ms_total * 1e-3)
+
+
 def layer_set_weights(cfg):
     return sum(L.c * L.b for L in cfg.layers)
 
@@ -207,10 +224,7 @@ def run_ours(args):
     launches = T.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     ms_total = t_start.elapsed_time(t_end)
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, dev)
     # device status of the last step
     for st in stats_last:
         ps = T.PruneStats.from_bytes(bytes(st.cpu().numpy().tobytes()))
@@ -219,7 +233,7 @@ def run_ours(args):
 
     nweights = layer_set_weights(cfg)
     ms_per_step = ms_total / args.steps
-    value = world * nweights * args.steps / (ms_total * 1e-3)
+    value = whole_job_rate(nweights, args.steps, world, ms_total)
 
     # ---- roofline of the dominant kernel: the Hessian contraction
     peaks = _peaks()
@@ -308,10 +322,7 @@ def run_e2e(T, cfg, a, dev, dt, margs, world, args):
         step()
     torch.cuda.synchronize()
     dt_s = time.perf_counter() - t0
-    if world > 1:
-        tt = torch.tensor([dt_s], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dt_s = float(tt.item())
+    dt_s = max_over_ranks(dt_s, dev)
     return {"value": world * layer_set_weights(cfg) * steps / dt_s, "unit": UNIT,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
             "ms_per_step": dt_s * 1e3 / steps}
@@ -400,6 +411,47 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_single_layer(args):
+    """One layer (c, b) with `a` calibration tokens through the three calls, `--reps` times; the
+    small, fixed command the ncu captures under profiles/ were taken with."""
+    import paper_2504_05346_b200 as T
+    from paper_2504_05346_b200 import build as B_
+
+    B_.build()
+    T.load_library()
+    c, b, a = [int(v) for v in args.single_layer.split(",")]
+    cfg = WL.CONFIGS[args.workload]
+    dev = torch.device("cuda", 0)
+    margs = mode_args(cfg, T)
+    W = WL.make_weight(c, b, cfg.dtype, seed=cfg.seed, layer_index=0, device=dev)
+    X = WL.make_activations(a, b, cfg.dtype, cfg.x_dist, cfg.outlier_frac, cfg.outlier_count,
+                            cfg.outlier_scale, cfg.seed, 0, device=dev)
+    H = torch.zeros((b, b), dtype=torch.float32, device=dev)
+    out = []
+    for _ in range(args.reps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        H.zero_()
+        ev[0].record()
+        T.hessian_accumulate(H, X)
+        ev[1].record()
+        if args.hessian_only:
+            torch.cuda.synchronize()
+            ms = ev[0].elapsed_time(ev[1])
+            out.append({"hessian_ms": round(ms, 4),
+                        "hessian_tflops": round(a * b * (b + 1.0) / ms / 1e9, 1)})
+            continue
+        U, xn = T.prepare_inverse(H, cfg.damp_rel)
+        ev[2].record()
+        _, _, st = T.prune_layer(W, U, xn, B=cfg.B, **margs)
+        ev[3].record()
+        torch.cuda.synchronize()
+        out.append({"hessian_ms": round(ev[0].elapsed_time(ev[1]), 4),
+                    "prepare_ms": round(ev[1].elapsed_time(ev[2]), 4),
+                    "prune_ms": round(ev[2].elapsed_time(ev[3]), 4), "n_pruned": st.n_pruned,
+                    "select_misses": st.select_misses})
+    print(json.dumps({"single_layer": [c, b, a], "workload": cfg.name, "runs": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -412,7 +464,14 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    ap.add_argument("--single-layer", default="", metavar="C,B,A",
+                    help="profile driver: one c x b layer with a tokens instead of the layer set")
+    ap.add_argument("--hessian-only", action="store_true", help="with --single-layer: stop after H")
+    ap.add_argument("--reps", type=int, default=1)
     args = ap.parse_args()
+    if args.single_layer:
+        run_single_layer(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
