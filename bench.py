@@ -32,6 +32,25 @@ UNIT = "weights/s"
 TOKEN_CHUNK = 262144  # tokens per thanos_hessian_accumulate call (the activations are resident)
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the Hessian kernel from
+# the ncu captures summarised under profiles/ (hessian_tc2_kernel_*.md): width b -> (bytes, tokens
+# of the captured launch).  A launch streams X once per wave of tile pairs, so its traffic grows in
+# proportion to its tokens; the figure reported with the bench line is scaled that way.
+HESSIAN_DRAM_CAPTURE = {4096: (2.083e9, 65536), 11008: (4.567e9, 16384)}
+
+
+def hessian_traffic_per_launch(launch_shapes):
+    """Average scaled DRAM bytes per launch over (b, tokens) launches; None if a width was never
+    captured."""
+    tot = 0.0
+    for b, tok in launch_shapes:
+        if b not in HESSIAN_DRAM_CAPTURE:
+            return None
+        byt, cap_tok = HESSIAN_DRAM_CAPTURE[b]
+        tot += byt * tok / cap_tok
+    return tot / max(1, len(launch_shapes))
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -180,7 +199,7 @@ def run_ours(args):
                 T.hessian_accumulate(H, xc, workspace=ws)
                 if record:
                     e.record()
-                    hess_events.append((s, e, float(xc.shape[0]) * b * (b + 1)))
+                    hess_events.append((s, e, float(xc.shape[0]) * b * (b + 1), (b, int(xc.shape[0]))))
             e1 = torch.cuda.Event(enable_timing=True)
             e1.record()
             U, xn = T.prepare_inverse(H, cfg.damp_rel, workspace=ws, check=False)
@@ -237,14 +256,17 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel: the Hessian contraction
     peaks = _peaks()
-    h_ms = sum(s.elapsed_time(e) for s, e, _ in hess_events)
-    h_flops = sum(f for _, _, f in hess_events)
+    h_ms = sum(ev[0].elapsed_time(ev[1]) for ev in hess_events)
+    h_flops = sum(ev[2] for ev in hess_events)
+    traffic = hessian_traffic_per_launch([ev[3] for ev in hess_events])
     achieved = h_flops / (h_ms * 1e-3) / 1e12 if h_ms > 0 else 0.0
     peak = peaks["bf16_tflops_sustained"]
     phase_ms = {k: sum(s.elapsed_time(e) for s, e in v) / args.steps for k, v in phase_events.items()}
-    roofline = {"kernel": "hessian_accumulate", "bound": "tensor", "achieved": round(achieved, 2),
+    roofline = {"kernel": "hessian_tc2_kernel (thanos_hessian_accumulate)", "bound": "tensor", "achieved": round(achieved, 2),
                 "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
-                "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None,
+                "peak_source": peaks["source"] + " (sustained bf16)",
+                "traffic": None if traffic is None else round(traffic),
+                "traffic_unit": "DRAM bytes per launch, ncu capture of a shorter launch scaled by tokens",
                 "launches": len(hess_events), "avg_launch_ms": round(h_ms / max(1, len(hess_events)), 4)}
 
     # ---- end to end through the host-buffer entry point
