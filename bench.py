@@ -170,54 +170,91 @@ def run_ours(args):
     weights = [WL.config_weight(cfg, i, device=dev) for i in range(len(cfg.layers))]
     outs = [torch.empty_like(w) for w in weights]
     masks = [torch.empty(w.shape, dtype=torch.uint8, device=dev) for w in weights]
-    bs = sorted({L.b for L in cfg.layers})
-    Hbuf = {b: torch.empty((b, b), dtype=torch.float32, device=dev) for b in bs}
-    ws_bytes = 256
-    for L in cfg.layers:
-        ws_bytes = max(ws_bytes, T.workspace_bytes(0, 0, L.b, 0, dt),
-                       T.workspace_bytes(1, 0, L.b, 0, T.F32),
-                       T.workspace_bytes(2, L.c, L.b, cfg.B, dt))
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
+    # Layers of a block are pruned independently of each other, so every distinct input gets a
+    # stream (Hessian + factorisation) and every layer a stream (sweep) with buffers of their own:
+    # the serial chains of small kernels of one call then fill the gaps of the others.
+    overlap = not args.no_overlap
+    main = torch.cuda.current_stream()
+    in_ids = list(inputs.keys())
+    s_in = {iid: (torch.cuda.Stream() if overlap else main) for iid in in_ids}
+    s_layer = [torch.cuda.Stream() if overlap else main for _ in cfg.layers]
+    Hbuf, Ubuf, xnbuf, ws_in = {}, {}, {}, {}
+    for iid in in_ids:
+        b = inputs[iid].shape[1]
+        Hbuf[iid] = torch.empty((b, b), dtype=torch.float32, device=dev)
+        Ubuf[iid] = torch.empty((b, b), dtype=torch.float32, device=dev)
+        xnbuf[iid] = torch.empty((b,), dtype=torch.float32, device=dev)
+        nb = max(T.workspace_bytes(0, 0, b, 0, dt), T.workspace_bytes(1, 0, b, 0, T.F32))
+        ws_in[iid] = torch.empty(nb, dtype=torch.uint8, device=dev)
+    ws_layer = [torch.empty(T.workspace_bytes(2, L.c, L.b, cfg.B, dt), dtype=torch.uint8, device=dev)
+                for L in cfg.layers]
+    torch.cuda.synchronize()
 
-    hess_events = []  # (start, end, flops) per thanos_hessian_accumulate call
+    hess_events = []  # (start, end, flops, (b, tokens)) per thanos_hessian_accumulate call
     phase_events = {"hessian": [], "prepare": [], "prune": []}
 
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
     def one_step(record):
-        stats_all = []
-        for iid, X in inputs.items():
+        stats_all = [None] * len(cfg.layers)
+        # the Hessians fill the whole GPU by themselves: one after the other on the main stream
+        for iid in in_ids:
+            X = inputs[iid]
             b = X.shape[1]
-            H = Hbuf[b]
-            e0 = torch.cuda.Event(enable_timing=True)
-            e0.record()
+            H = Hbuf[iid]
+            e0 = ev()
+            e0.record(main)
             H.zero_()
             for t0 in range(0, a, TOKEN_CHUNK):
                 xc = X[t0:t0 + TOKEN_CHUNK]
                 if record:
-                    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    s.record()
-                T.hessian_accumulate(H, xc, workspace=ws)
+                    hs, he = ev(), ev()
+                    hs.record(main)
+                T.hessian_accumulate(H, xc, workspace=ws_in[iid])
                 if record:
-                    e.record()
-                    hess_events.append((s, e, float(xc.shape[0]) * b * (b + 1), (b, int(xc.shape[0]))))
-            e1 = torch.cuda.Event(enable_timing=True)
-            e1.record()
-            U, xn = T.prepare_inverse(H, cfg.damp_rel, workspace=ws, check=False)
-            e2 = torch.cuda.Event(enable_timing=True)
-            e2.record()
-            for i, L in enumerate(cfg.layers):
-                if L.input_id != iid:
-                    continue
-                _, _, st = T.prune_layer(weights[i], U, xn, B=cfg.B, workspace=ws, out=outs[i],
-                                         mask=masks[i], read_stats=False, **margs)
-                stats_all.append(st)
-            e3 = torch.cuda.Event(enable_timing=True)
-            e3.record()
+                    he.record(main)
+                    hess_events.append((hs, he, float(xc.shape[0]) * b * (b + 1),
+                                        (b, int(xc.shape[0]))))
+            e1 = ev()
+            e1.record(main)
             if record:
                 phase_events["hessian"].append((e0, e1))
+        e_h = ev()
+        e_h.record(main)
+        # factorisations and sweeps: one stream per input, then one per layer
+        ready = {}
+        for iid in in_ids:
+            s = s_in[iid]
+            s.wait_event(e_h)
+            with torch.cuda.stream(s):
+                e1 = ev()
+                e1.record(s)
+                T.prepare_inverse(Hbuf[iid], cfg.damp_rel, workspace=ws_in[iid], check=False,
+                                  factor=Ubuf[iid], xnorm=xnbuf[iid])
+                e2 = ev()
+                e2.record(s)
+                ready[iid] = e2
+            if record:
                 phase_events["prepare"].append((e1, e2))
-                phase_events["prune"].append((e2, e3))
-            del U, xn
+        done = []
+        for i, L in enumerate(cfg.layers):
+            s = s_layer[i]
+            s.wait_event(ready[L.input_id])
+            with torch.cuda.stream(s):
+                p0 = ev()
+                p0.record(s)
+                _, _, st = T.prune_layer(weights[i], Ubuf[L.input_id], xnbuf[L.input_id], B=cfg.B,
+                                         workspace=ws_layer[i], out=outs[i], mask=masks[i],
+                                         read_stats=False, **margs)
+                p1 = ev()
+                p1.record(s)
+            stats_all[i] = st
+            done.append(p1)
+            if record:
+                phase_events["prune"].append((p0, p1))
+        for e in done:
+            main.wait_event(e)
         return stats_all
 
     def barrier():
@@ -291,6 +328,8 @@ def run_ours(args):
                                       cfg.B, cfg.damp_rel),
                        "weights_per_step": nweights, "l2": "inputs larger than L2",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "streams": ("one per layer input and one per layer (calls overlap; "
+                                   "phase_ms_per_step sums per-call times)") if overlap else "one",
                        "token_chunk": TOKEN_CHUNK},
             "ms_per_layer": ms_per_step / len(cfg.layers),
             "phase_ms_per_step": {k: round(v, 3) for k, v in phase_ms.items()},
@@ -483,6 +522,8 @@ def main():
     ap.add_argument("--workload", default="llama2_7b", choices=sorted(WL.CONFIGS))
     ap.add_argument("--tokens", type=int, default=0, help="override the calibration token count")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="issue every call on one stream instead of one stream per input / layer")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)

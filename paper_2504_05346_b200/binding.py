@@ -175,14 +175,19 @@ def hessian_accumulate(H: torch.Tensor, X: torch.Tensor, stream=None,
 
 
 def prepare_inverse(H: torch.Tensor, damp_rel: float, stream=None,
-                    workspace: Optional[torch.Tensor] = None,
-                    check: bool = True) -> Tuple[torch.Tensor, torch.Tensor]:
-    """Returns (factor U [b, b] upper-triangular with U^T U = (H + damp I)^-1, xnorm [b])."""
+                    workspace: Optional[torch.Tensor] = None, check: bool = True,
+                    factor: Optional[torch.Tensor] = None,
+                    xnorm: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Returns (factor U [b, b] upper-triangular with U^T U = (H + damp I)^-1, xnorm [b]);
+    pass `factor` / `xnorm` to have them written into existing buffers."""
     lib = load_library()
     _check_dev(H)
     b = H.shape[0]
-    factor = torch.empty((b, b), dtype=torch.float32, device=H.device)
-    xnorm = torch.empty((b,), dtype=torch.float32, device=H.device)
+    if factor is None:
+        factor = torch.empty((b, b), dtype=torch.float32, device=H.device)
+    if xnorm is None:
+        xnorm = torch.empty((b,), dtype=torch.float32, device=H.device)
+    _check_dev(factor, xnorm)
     status = torch.zeros(4, dtype=torch.int32, device=H.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_PREPARE, 0, b, 0, F32), H.device)

@@ -71,10 +71,10 @@ def test_hessian_strided_input_and_empty_chunk(T):
     assert PU.rel_fro(_np64(H), Ho) <= PU.TOL_H
 
 
-def test_hessian_bench_shape_sampled(T):
-    """b = 4096 with a 32768-token bf16 chunk (the benchmark's launch shape): sampled entries
-    against a float64 dot product."""
-    b, n_tok = 4096, 32768
+@pytest.mark.parametrize("b,n_tok", [(4096, 32768), (11008, 12345)])
+def test_hessian_bench_shape_sampled(T, b, n_tok):
+    """The benchmark's layer widths with long bf16 chunks (CTA-pair kernel, several token slices,
+    a ragged token tail): sampled entries against a float64 dot product."""
     Xd = WL.make_activations(n_tok, b, "bf16", "student_t4", 0.005, 0, 50.0, 2, 0, device=DEV)
     H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
     T.hessian_accumulate(H, Xd)
