@@ -344,6 +344,7 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
       g.N = N;
       g.K = N;
       g.batch = part == 0 ? cnt : 1;
+      g.b_upper = 1;  // U22 is upper-triangular
       g.status = w.tc_status;
       THANOS_TRY(tc_gemm_split3(g, stream));
       TcGemmArgs h;
@@ -367,6 +368,7 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
       h.N = N;
       h.K = (int)sz;
       h.batch = part == 0 ? cnt : 1;
+      h.a_upper = 1;  // U11 is upper-triangular
       h.alpha = -1.f;
       h.status = w.tc_status;
       THANOS_TRY(tc_gemm_split3(h, stream));

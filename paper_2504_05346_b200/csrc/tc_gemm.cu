@@ -41,7 +41,7 @@ struct Params {
   int32_t* status;
   int M, N, K, batch;
   int tiles_m, tiles_n;
-  int b_kmajor, accumulate, upper_only;
+  int b_kmajor, accumulate, upper_only, a_upper, b_upper;
   float alpha;
 };
 
@@ -108,6 +108,7 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads) {
 
 struct Tile {
   int z, m0, n0;
+  int ks0, ks1;  // k steps [ks0, ks1) that can hold non-zero products
   bool skip;
 };
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t) {
@@ -119,6 +120,13 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t) {
   r.m0 = mi * TM;
   r.n0 = (rem - mi * p.tiles_n) * TN;
   r.skip = p.upper_only && (r.n0 + TN - 1 < r.m0);
+  r.ks0 = p.a_upper ? r.m0 / BK : 0;
+  r.ks1 = (p.K + BK - 1) / BK;
+  if (p.b_upper) {
+    const int lim = (r.n0 + TN + BK - 1) / BK;
+    if (lim < r.ks1) r.ks1 = lim;
+  }
+  if (r.ks1 <= r.ks0) r.ks1 = r.ks0 + 1;  // at least one step so that the accumulator is defined
   return r;
 }
 
@@ -170,7 +178,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int n_tiles = p.tiles_m * p.tiles_n * p.batch;
-  const int ksteps = (p.K + BK - 1) / BK;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -180,7 +187,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
       const Tile tl = decode_tile(p, t);
       if (tl.skip) continue;
-      for (int ks = 0; ks < ksteps && ok; ++ks) {
+      for (int ks = tl.ks0; ks < tl.ks1 && ok; ++ks) {
         ok = mbar_wait(empty_bar(s), phase ^ 1u, abort_flag);
         if (ok && lane == 0) {
           const uint32_t dst = smem_base + (uint32_t)s * STAGE_BYTES;
@@ -226,7 +233,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       if (tl.skip) continue;
       ok = mbar_wait(tempty_bar(q), tphase ^ 1u, abort_flag);
       tc_fence_after();
-      for (int ks = 0; ks < ksteps && ok; ++ks) {
+      for (int ks = tl.ks0; ks < tl.ks1 && ok; ++ks) {
         ok = mbar_wait(full_bar(s), phase, abort_flag);
         tc_fence_after();
         if (ok && lane == 0) {
@@ -242,7 +249,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
               const uint64_t bdesc =
                   p.b_kmajor ? desc_kmajor(pb + k4 * 32) : desc_mnmajor(pb + k4 * 2048);
               tc_mma_bf16(tmem_base + (uint32_t)q * TN, adesc, bdesc, idesc,
-                          (ks > 0 || cb > 0 || k4 > 0) ? 1u : 0u);
+                          (ks > tl.ks0 || cb > 0 || k4 > 0) ? 1u : 0u);
             }
           }
           tc_commit(empty_bar(s));
@@ -474,6 +481,8 @@ thanos_status_t tc_gemm_split3(const TcGemmArgs& a, cudaStream_t stream) {
   p.b_kmajor = a.b_kmajor;
   p.accumulate = a.accumulate;
   p.upper_only = a.upper_only;
+  p.a_upper = a.a_upper;
+  p.b_upper = a.b_upper;
   p.alpha = a.alpha;
   const long long tiles = (long long)p.tiles_m * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return THANOS_ERR_SHAPE;

@@ -32,6 +32,8 @@ struct TcGemmArgs {
   float alpha = 1.f;
   int accumulate = 0;
   int upper_only = 0;            // skip tiles that lie strictly below the diagonal (n0 + 127 < m0)
+  int a_upper = 0;               // A[m, k] = 0 for k < m: a tile starts its k loop at its first row
+  int b_upper = 0;               // Bop[k, n] = 0 for k > n: a tile ends its k loop at its last column
   int32_t* status = nullptr;     // device int32: THANOS_ERR_TIMEOUT if a bounded wait ran out
 };
 
