@@ -30,8 +30,9 @@ namespace {
 // the running budget r of Algorithm 1).  Keys are the fp32 bit patterns of |w| * ||X_j|| (>= 0, so
 // they order like the values).  Two routes, both exact:
 //   bracket  the threshold moves little from block to block, so one pass counts the keys below a
-//            window of 2^18 key values around the previous threshold and bins the keys inside it
-//            (512 bins of 512 values); a second pass resolves the 512 values of the hit bin;
+//            window of 2^18 key values around the previous threshold, bins the keys inside it
+//            (512 bins of 512 values) and copies them out (about 3 in 100); a second, short pass
+//            over the copied keys resolves the 512 values of the hit bin;
 //   radix    four passes over 8, 8, 8 and 7 key bits (first block, or when the window misses).
 // One kernel, launched five times per block, does whichever pass the sweep state asks for; the
 // last CTA to finish a pass reads the histogram, decides and sets the next phase.
@@ -40,6 +41,7 @@ constexpr int RADIX_BINS = 256;
 constexpr int RADIX_REPL = 8;           // shared-memory copies of a radix histogram (by lane & 7)
 constexpr unsigned WINDOW = 1u << 18;   // key values covered by the bracket
 constexpr int WINDOW_SHIFT = 9;         // 512 values per bracket bin
+constexpr int CTA_CAND = 6144;          // keys inside the window one CTA can hold before copying out
 __host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0)); }
 
@@ -64,6 +66,8 @@ struct SweepState {
   int phase;                     // what the next select pass does
   unsigned int ticket;           // CTAs that have finished the current pass
   unsigned int mark_ticket;      // same for the mask kernel
+  unsigned int cand_total;       // keys the bracket pass copied out of its window
+  int cand_overflow;             // the copy did not fit: the refine pass rescans the residual
   int pad;
 };
 
@@ -223,8 +227,11 @@ __device__ __forceinline__ void find_rank_bin(const unsigned* hist, int nbin, un
 __global__ void __launch_bounds__(256)
 select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                    int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
-                   unsigned* __restrict__ list_counts, int first_launch, thanos_stats_t* stats) {
+                   unsigned* __restrict__ list_counts, int first_launch, thanos_stats_t* stats,
+                   unsigned* __restrict__ cand, unsigned cand_cap) {
   __shared__ unsigned sh[RADIX_BINS * RADIX_REPL];
+  __shared__ unsigned s_cand[CTA_CAND];
+  __shared__ unsigned s_ncand, s_cbase;
   __shared__ int s_last;
   __shared__ unsigned s_below;
   const int phase = st->phase;
@@ -239,7 +246,10 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
   const bool radix = phase <= PH_RADIX3;
   const int nclear = radix ? RADIX_BINS * RADIX_REPL : HIST_BINS;
   for (int i = threadIdx.x; i < nclear; i += 256) sh[i] = 0;
-  if (threadIdx.x == 0) s_below = 0;
+  if (threadIdx.x == 0) {
+    s_below = 0;
+    s_ncand = 0;
+  }
   __syncthreads();
   unsigned below = 0;
   if (radix) {
@@ -269,30 +279,49 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
         }
       }
     }
+  } else if (phase == PH_REFINE && !st->cand_overflow) {
+    // the bracket pass copied every key of its window out: only those are looked at again
+    const unsigned lo = st->lo;
+    const unsigned total = st->cand_total;
+    for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total; i += gridDim.x * 256u) {
+      const unsigned d = __ldcg(&cand[i]) - lo;
+      if (d < (unsigned)HIST_BINS) atomicAdd(&sh[d], 1u);
+    }
   } else {
     const unsigned lo = st->lo;
-    const unsigned width = phase == PH_BRACKET ? WINDOW : (unsigned)HIST_BINS;
-    const int bshift = phase == PH_BRACKET ? WINDOW_SHIFT : 0;
+    const bool bracket = phase == PH_BRACKET;
+    const unsigned width = bracket ? WINDOW : (unsigned)HIST_BINS;
+    const int bshift = bracket ? WINDOW_SHIFT : 0;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-      for (int q0 = threadIdx.x; q0 < w4; q0 += 4 * 256) {
+      for (int qb = 0; qb < w4; qb += 4 * 256) {
+        const int q0 = qb + (int)threadIdx.x;
         float4 w[4], x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {  // four loads in flight per thread
           const int q = q0 + u * 256;
           w[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
-          x[u] = q < w4 ? __ldg(&xr[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[u] = q < w4 ? __ldg(&xr[q]) : make_float4(1.f, 1.f, 1.f, 1.f);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          if (q0 + u * 256 >= w4) break;
+          // lanes past the row's end carry key 0 < lo or fall outside the window: handled below
+          const bool live = q0 + u * 256 < w4;
           const unsigned k[4] = {metric_key(w[u].x, x[u].x), metric_key(w[u].y, x[u].y),
                                  metric_key(w[u].z, x[u].z), metric_key(w[u].w, x[u].w)};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const unsigned d = k[e] - lo;
-            if (k[e] < lo) ++below;
-            else if (d < width) atomicAdd(&sh[d >> bshift], 1u);
+            if (!live) continue;
+            if (k[e] < lo) {
+              ++below;
+            } else if (d < width) {
+              atomicAdd(&sh[d >> bshift], 1u);
+              if (bracket) {  // copy the key out (about three keys in a hundred get here)
+                const unsigned pos = atomicAdd(&s_ncand, 1u);
+                if (pos < (unsigned)CTA_CAND) s_cand[pos] = k[e];
+              }
+            }
           }
         }
       }
@@ -314,7 +343,21 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       for (int o = 16; o > 0; o >>= 1) below += __shfl_down_sync(0xffffffffu, below, o);
       if (lane == 0 && below) atomicAdd(&s_below, below);
       __syncthreads();
-      if (threadIdx.x == 0 && s_below) atomicAdd(&st->below, (unsigned long long)s_below);
+      const unsigned ncand = s_ncand;
+      if (threadIdx.x == 0) {
+        if (s_below) atomicAdd(&st->below, (unsigned long long)s_below);
+        if (ncand > (unsigned)CTA_CAND) {
+          st->cand_overflow = 1;
+          s_cbase = cand_cap;
+        } else {
+          s_cbase = ncand ? atomicAdd(&st->cand_total, ncand) : 0u;
+          if (ncand && s_cbase + ncand > cand_cap) st->cand_overflow = 1;
+        }
+      }
+      __syncthreads();
+      const unsigned cbase = s_cbase;
+      if (ncand <= (unsigned)CTA_CAND && cbase + ncand <= cand_cap)
+        for (unsigned i = threadIdx.x; i < ncand; i += 256) cand[cbase + i] = s_cand[i];
     }
   }
   // ---- the last CTA to get here decides
@@ -394,6 +437,10 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     st->below = 0;
     st->ticket = 0;
     st->phase = next;
+    if (next != PH_REFINE) {  // the copied keys are only needed by the refine pass
+      st->cand_total = 0;
+      st->cand_overflow = 0;
+    }
   }
 }
 
@@ -609,9 +656,19 @@ struct SweepWs {
   SweepState* st;
   unsigned* rowcnt;
   unsigned long long* rowbase;
+  unsigned* cand;         // keys copied out of the bracket window
+  size_t cand_cap;
   int* row_lists;         // [2, c] rows of the current block by kind of system
   unsigned* list_counts;  // [2]
 };
+
+// room for one key in eight of the layer (the bracket window holds about three in a hundred)
+size_t cand_capacity(int64_t c, int64_t b) {
+  size_t n = (size_t)c * (size_t)b / 8;
+  if (n < 4096) n = 4096;
+  if (n > ((size_t)1 << 31)) n = (size_t)1 << 31;
+  return n;
+}
 
 bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, int32_t B,
            bool need_wc) {
@@ -629,6 +686,8 @@ bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, i
   w.st = ar.take<SweepState>(1);
   w.rowcnt = ar.take<unsigned>((size_t)c);
   w.rowbase = ar.take<unsigned long long>((size_t)c);
+  w.cand_cap = cand_capacity(c, b);
+  w.cand = ar.take<unsigned>(w.cand_cap);
   w.row_lists = ar.take<int>(2 * (size_t)c);
   w.list_counts = ar.take<unsigned>(2);
   return ar.ok();
@@ -665,8 +724,11 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < 148 * 4 ? c : 148 * 4;
     for (int pass = 0; pass < 5; ++pass) {
-      select_pass_kernel<<<sg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
-                                                 w.list_counts, pass == 0 ? 1 : 0, stats);
+      // passes after the first usually look at the copied keys only, or do nothing
+      const int sgp = pass == 0 ? sg : (sg < 148 * 2 ? sg : 148 * 2);
+      select_pass_kernel<<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                 w.list_counts, pass == 0 ? 1 : 0, stats, w.cand,
+                                                 (unsigned)w.cand_cap);
       THANOS_CHECK_LAUNCH();
     }
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
@@ -725,6 +787,7 @@ size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dty
   t += round_up((size_t)c * sizeof(unsigned), 256);
   t += round_up((size_t)c * sizeof(unsigned long long), 256);
   t += round_up(2 * (size_t)c * sizeof(int), 256);
+  t += round_up(cand_capacity(c, b) * sizeof(unsigned), 256);
   t += 256;
   return t + 256;
 }
