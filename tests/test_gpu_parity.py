@@ -481,6 +481,26 @@ def test_full_size_layer_sampled_rows(T):
         assert PU.rel_fro(_np64(Wp)[rows], Wr) <= PU.TOL_W_BF16
 
 
+def test_wide_layer_11008_sampled_rows(T):
+    """The down-projection width of the benchmark (b = 11008, 86 blocks of 128) with fewer rows:
+    counts, exact zeros, and a float64 replay of sampled rows under the GPU's mask."""
+    c, b, B = 512, 11008, 128
+    W = WL.make_weight(c, b, "bf16", seed=2, layer_index=6, device=DEV)
+    Xd = WL.make_activations(12288, b, "bf16", "student_t4", 0.005, 0, 50.0, 2, 3, device=DEV)
+    H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(H, Xd)
+    U, xn = T.prepare_inverse(H, 0.01)
+    Wp, M, st = T.prune_layer(W, U, xn, T.UNSTRUCTURED, p=0.5, B=B)
+    assert st.n_pruned == c * b // 2 and st.r_left == 0 and st.n_blocks == b // B
+    assert st.select_misses <= 2
+    assert bool((Wp[M.bool()] == 0).all())
+    Hd = O.damped(_np64(H), 0.01)
+    rows = np.array([0, 255, 511])
+    Wr = O.replay_rows(_np64(W)[rows], M.cpu().numpy()[rows], Hd, B)
+    Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
+    assert PU.rel_fro(_np64(Wp)[rows], Wr) <= PU.TOL_W_BF16
+
+
 def test_host_buffer_entry_point_matches_device_path(T):
     c, b, a, B = 96, 256, 20000, 64
     W = WL.make_weight(c, b, "bf16", seed=61)
