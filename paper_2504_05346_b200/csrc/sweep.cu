@@ -287,42 +287,49 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       const unsigned d = __ldcg(&cand[i]) - lo;
       if (d < (unsigned)HIST_BINS) atomicAdd(&sh[d], 1u);
     }
-  } else {
+  } else if (phase == PH_BRACKET) {
+    // The hot pass: per element one multiply, one compare-and-count, one window test; keys inside
+    // the window (about 3 in 100) take the slow path that bins and copies them.
     const unsigned lo = st->lo;
-    const bool bracket = phase == PH_BRACKET;
-    const unsigned width = bracket ? WINDOW : (unsigned)HIST_BINS;
-    const int bshift = bracket ? WINDOW_SHIFT : 0;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-      for (int qb = 0; qb < w4; qb += 4 * 256) {
-        const int q0 = qb + (int)threadIdx.x;
-        float4 w[4], x[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {  // four loads in flight per thread
-          const int q = q0 + u * 256;
-          w[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
-          x[u] = q < w4 ? __ldg(&xr[q]) : make_float4(1.f, 1.f, 1.f, 1.f);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          // lanes past the row's end carry key 0 < lo or fall outside the window: handled below
-          const bool live = q0 + u * 256 < w4;
-          const unsigned k[4] = {metric_key(w[u].x, x[u].x), metric_key(w[u].y, x[u].y),
-                                 metric_key(w[u].z, x[u].z), metric_key(w[u].w, x[u].w)};
+#pragma unroll 2
+      for (int q = threadIdx.x; q < w4; q += 256) {
+        const float4 w = wr[q];
+        const float4 x = __ldg(&xr[q]);
+        const unsigned k0 = metric_key(w.x, x.x), k1 = metric_key(w.y, x.y);
+        const unsigned k2 = metric_key(w.z, x.z), k3 = metric_key(w.w, x.w);
+        below += (k0 < lo) + (k1 < lo) + (k2 < lo) + (k3 < lo);
+        // k - lo wraps to a huge value for k < lo, so one unsigned test finds the window
+        const unsigned d0 = k0 - lo, d1 = k1 - lo, d2 = k2 - lo, d3 = k3 - lo;
+        if ((d0 < WINDOW) | (d1 < WINDOW) | (d2 < WINDOW) | (d3 < WINDOW)) {
+          const unsigned kk[4] = {k0, k1, k2, k3};
+          const unsigned dd[4] = {d0, d1, d2, d3};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const unsigned d = k[e] - lo;
-            if (!live) continue;
-            if (k[e] < lo) {
-              ++below;
-            } else if (d < width) {
-              atomicAdd(&sh[d >> bshift], 1u);
-              if (bracket) {  // copy the key out (about three keys in a hundred get here)
-                const unsigned pos = atomicAdd(&s_ncand, 1u);
-                if (pos < (unsigned)CTA_CAND) s_cand[pos] = k[e];
-              }
+            if (dd[e] < WINDOW) {
+              atomicAdd(&sh[dd[e] >> WINDOW_SHIFT], 1u);
+              const unsigned pos = atomicAdd(&s_ncand, 1u);
+              if (pos < (unsigned)CTA_CAND) s_cand[pos] = kk[e];
             }
           }
+        }
+      }
+    }
+  } else {
+    // refine over the whole residual (only when the copied keys did not fit)
+    const unsigned lo = st->lo;
+    for (int row = blockIdx.x; row < c; row += gridDim.x) {
+      const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+      for (int q = threadIdx.x; q < w4; q += 256) {
+        const float4 w = wr[q];
+        const float4 x = __ldg(&xr[q]);
+        const unsigned k[4] = {metric_key(w.x, x.x), metric_key(w.y, x.y), metric_key(w.z, x.z),
+                               metric_key(w.w, x.w)};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned d = k[e] - lo;
+          if (d < (unsigned)HIST_BINS) atomicAdd(&sh[d], 1u);
         }
       }
     }
