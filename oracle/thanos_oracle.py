@@ -220,20 +220,58 @@ def thanos_unstructured(W, X, p, B, damp_rel=0.0, H=None, collect=None):
     return Wp, M, H
 
 
-def thanos_nm(W, X, n, m, B, damp_rel=0.0, H=None, collect=None):
-    """Algorithm 4 with ``alpha = 0`` (no outlier rows, identity row permutation)."""
+def row_losses(W, X=None, H=None):
+    """``h_i = ||W_i X||_2^2``: the loss of Eq. 1 when row ``i`` is removed entirely (definition
+    of the outlier rows, Section 4.7).  From the Hessian it is ``1/2 W_i H W_i^T``."""
+    W = np.asarray(W, dtype=F64)
+    if X is not None:
+        return np.sum((W @ np.asarray(X, dtype=F64)) ** 2, axis=1)
+    return 0.5 * np.einsum("ij,jk,ik->i", W, np.asarray(H, dtype=F64), W)
+
+
+def outlier_row_order(h, alpha):
+    """Row permutation of Algorithm 4: rows in ascending order of ``h`` (stable: equal losses keep
+    their row order), so the ``ceil(alpha c)`` outlier rows come last.  Returns
+    ``(sigma, n_out)`` with ``sigma[k]`` = original index of the row at position ``k``.
+
+    Reading: the section defining alpha fixes the number of outlier rows as ``ceil(alpha c)``; the
+    listing's row loop runs to ``ceil(c (1 - alpha))``, which is one more row when ``alpha c`` is
+    not an integer.  The count from the definition is used: ``c - ceil(alpha c)`` rows are pruned.
+    """
+    h = np.asarray(h, dtype=F64)
+    c = h.shape[0]
+    n_out = int(math.ceil(float(alpha) * c - 1e-12)) if alpha > 0 else 0
+    sigma = np.argsort(h, kind="stable")
+    return sigma, n_out
+
+
+def thanos_nm(W, X, n, m, B, damp_rel=0.0, H=None, collect=None, alpha=0.0):
+    """Algorithm 4.  ``alpha`` is the fraction of outlier rows: the ``ceil(alpha c)`` rows with the
+    largest ``h_i = ||W_i X||^2`` are moved last by the row permutation ``Q`` and are not pruned;
+    the inverse permutation restores the row order at the end."""
     W = np.asarray(W, dtype=F64)
     if B % m != 0:
         raise ValueError("block size B must be a multiple of m")
     if H is None:
         H = hessian(X)
     xn = feature_norms(H)
+    c = W.shape[0]
+    if alpha > 0:
+        sigma, n_out = outlier_row_order(row_losses(W, H=H), alpha)
+    else:
+        sigma, n_out = np.arange(c), 0
+    Wq = W[sigma]                      # W <- Q W
+    n_pruned_rows = c - n_out
 
     def block_mask(Wc, j1, j2):
-        return nm_block_mask(Wc[:, j1:j2], xn[j1:j2], n, m)
+        Mb = nm_block_mask(Wc[:, j1:j2], xn[j1:j2], n, m)
+        Mb[n_pruned_rows:] = 0         # the row loop of the listing stops before the outliers
+        return Mb
 
-    Wp, M = _sweep(W, H, xn, B, damp_rel, block_mask, collect)
-    return Wp, M, H
+    Wp, M = _sweep(Wq, H, xn, B, damp_rel, block_mask, collect)
+    inv = np.empty(c, dtype=np.int64)
+    inv[sigma] = np.arange(c)
+    return Wp[inv], M[inv], H          # W <- Q^T W
 
 
 # --------------------------------------------------------------------------------------

@@ -344,3 +344,43 @@ def test_ragged_last_block_and_p_zero():
     assert int(M.sum()) == math.floor(0.3 * c * b)
     Wp0, M0, _ = O.thanos_unstructured(W, X, 0.0, 4, 0.01)
     assert M0.sum() == 0 and np.array_equal(Wp0, W)
+
+
+# ------------------------------------------------------------------------------ outlier rows
+def test_row_losses_match_their_definition_and_the_hessian_form():
+    rng = np.random.default_rng(5)
+    W = rng.standard_normal((7, 12))
+    X = rng.standard_normal((12, 40))
+    h_def = np.array([np.linalg.norm(W[i] @ X) ** 2 for i in range(7)])   # ||W_i X||_2^2
+    assert np.allclose(O.row_losses(W, X=X), h_def, rtol=1e-12)
+    assert np.allclose(O.row_losses(W, H=O.hessian(X)), h_def, rtol=1e-12)
+    # removing row i entirely costs exactly h_i in the objective of Eq. 1
+    for i in (0, 3):
+        Wh = W.copy()
+        Wh[i] = 0.0
+        assert abs(O.objective(Wh, W, X) - h_def[i]) <= 1e-9 * h_def[i]
+
+
+def test_outlier_rows_are_the_largest_losses_and_stay_untouched():
+    rng = np.random.default_rng(6)
+    c, b, B = 10, 16, 8
+    W = rng.standard_normal((c, b))
+    X = rng.standard_normal((b, 64))
+    W[2] *= 30.0
+    W[7] *= 20.0                                   # two rows with by far the largest h_i
+    alpha = 0.15                                   # ceil(1.5) = 2 outlier rows
+    Wp, M, H = O.thanos_nm(W, X, 2, 4, B, 0.01, alpha=alpha)
+    h = O.row_losses(W, X=X)
+    sigma, n_out = O.outlier_row_order(h, alpha)
+    assert n_out == 2 and set(sigma[-2:]) == {2, 7}
+    assert np.array_equal(Wp[[2, 7]], W[[2, 7]]) and M[[2, 7]].sum() == 0
+    # the other rows are pruned exactly as without outliers: rows are independent in n:m mode
+    W0, M0, _ = O.thanos_nm(W, X, 2, 4, B, 0.01)
+    keep = np.array([i for i in range(c) if i not in (2, 7)])
+    assert np.array_equal(M[keep], M0[keep]) and np.allclose(Wp[keep], W0[keep], rtol=0, atol=1e-12)
+    assert int(M.sum()) == (c - 2) * b // 2
+    # alpha = 0 is the plain algorithm; ties in h keep row order (stable)
+    Wz, Mz, _ = O.thanos_nm(W, X, 2, 4, B, 0.01, alpha=0.0)
+    assert np.array_equal(Mz, M0) and np.array_equal(Wz, W0)
+    s2, n2 = O.outlier_row_order(np.array([1.0, 3.0, 3.0, 0.5]), 0.25)
+    assert n2 == 1 and list(s2) == [3, 0, 1, 2]    # of the tied rows 1 and 2, row 2 is the outlier
