@@ -54,7 +54,8 @@ typedef enum {
   THANOS_WS_HESSIAN = 0,
   THANOS_WS_PREPARE = 1,
   THANOS_WS_PRUNE = 2,
-  THANOS_WS_HOST_LAYER = 3
+  THANOS_WS_HOST_LAYER = 3,
+  THANOS_WS_PRUNE_OUTLIERS = 4
 } thanos_ws_which_t;
 
 /* Per-call statistics and device-side status of thanos_prune_layer / thanos_prune_block,
@@ -142,6 +143,29 @@ thanos_status_t thanos_prune_layer(const void* W_in, void* W_out, uint8_t* mask_
                                    const float* factor, const float* xnorm, thanos_mode_t mode,
                                    double p, int32_t n, int32_t m, int32_t B, void* workspace,
                                    size_t ws_bytes, thanos_stats_t* stats_dev, void* stream);
+
+/*
+ * n:m sweep with outlier rows (Algorithm 4 with alpha > 0; outlier rows are defined in
+ * Section 4.7): h_i = ||W_i X||_2^2 = 1/2 W_i H W_i^T is the loss of removing row i entirely; the
+ * ceil(alpha c) rows with the largest h_i are left untouched (no entry removed, no update), every
+ * other row is pruned exactly as by thanos_prune_layer in mode THANOS_NM.  The listing moves the
+ * outlier rows last by a row permutation and undoes it at the end; rows are independent in n:m
+ * mode, so this call skips them in place instead.  Equal losses are ordered by row index (the
+ * higher index counts as the larger loss).
+ *
+ *  H        device fp32 [b, b], the UNDAMPED Hessian the factor was made from (full storage).
+ *  alpha    0 <= alpha < 1; c - ceil(alpha c) rows are pruned.
+ *  row_outlier_out  device uint8 [c] or NULL: 1 for the outlier rows.
+ *  workspace: thanos_workspace_bytes(THANOS_WS_PRUNE_OUTLIERS, c, b, B, wdtype) bytes.
+ * Everything else as in thanos_prune_layer.
+ */
+thanos_status_t thanos_prune_layer_outliers(const void* W_in, void* W_out, uint8_t* mask_out,
+                                            thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                            const float* factor, const float* xnorm,
+                                            const float* H, int32_t n, int32_t m, int32_t B,
+                                            double alpha, uint8_t* row_outlier_out,
+                                            void* workspace, size_t ws_bytes,
+                                            thanos_stats_t* stats_dev, void* stream);
 
 /*
  * One block step of the sweep from a caller-supplied state (the body of the block loop of

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     prune_layer_host,
     prune_layer_noalloc,
     dense_product,
+    prune_layer_outliers,
     workspace_bytes,
     launch_count,
     status_string,

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 
 F32, BF16 = 0, 1
 UNSTRUCTURED, NM = 0, 1
-WS_HESSIAN, WS_PREPARE, WS_PRUNE, WS_HOST_LAYER = 0, 1, 2, 3
+WS_HESSIAN, WS_PREPARE, WS_PRUNE, WS_HOST_LAYER, WS_PRUNE_OUTLIERS = 0, 1, 2, 3, 4
 
 
 class ThanosError(RuntimeError):
@@ -85,6 +85,9 @@ def load_library():
     lib.thanos_prune_layer.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, i32, ctypes.c_double,
                                        i32, i32, i32, vp, sz, vp, vp]
     lib.thanos_prune_layer.restype = i32
+    lib.thanos_prune_layer_outliers.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp, i32, i32, i32,
+                                                ctypes.c_double, vp, vp, sz, vp, vp]
+    lib.thanos_prune_layer_outliers.restype = i32
     lib.thanos_prune_block.argtypes = [vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i64, vp, vp,
                                        sz, vp, vp]
     lib.thanos_prune_block.restype = i32
@@ -340,3 +343,32 @@ def dense_product(A: torch.Tensor, B: torch.Tensor, b_transposed: bool = False, 
         if st != 0:
             raise ThanosError(st, "thanos_dense_product (device)")
     return out
+
+
+def prune_layer_outliers(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tensor,
+                         H: torch.Tensor, n: int, m: int, alpha: float, B: int = 128, stream=None,
+                         workspace: Optional[torch.Tensor] = None,
+                         out: Optional[torch.Tensor] = None, mask: Optional[torch.Tensor] = None):
+    """thanos_prune_layer_outliers: n:m sweep that leaves the ceil(alpha c) rows with the largest
+    h_i = 1/2 W_i H W_i^T untouched.  Returns (W_pruned, mask, outlier flags uint8 [c], stats)."""
+    lib = load_library()
+    _check_dev(W, factor, xnorm, H)
+    c, b = W.shape
+    dt = _dtype_code(W)
+    if out is None:
+        out = torch.empty_like(W)
+    if mask is None:
+        mask = torch.empty((c, b), dtype=torch.uint8, device=W.device)
+    flags = torch.empty((c,), dtype=torch.uint8, device=W.device)
+    stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
+    if workspace is None:
+        workspace = _ws(workspace_bytes(WS_PRUNE_OUTLIERS, c, b, B, dt), W.device)
+    _check(lib.thanos_prune_layer_outliers(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
+                                           factor.data_ptr(), xnorm.data_ptr(), H.data_ptr(), n, m,
+                                           B, float(alpha), flags.data_ptr(), workspace.data_ptr(),
+                                           workspace.numel(), stats.data_ptr(),
+                                           _stream_ptr(stream)), "thanos_prune_layer_outliers")
+    st = _read_stats(stats)
+    if st.status != 0:
+        raise ThanosError(st.status, "thanos_prune_layer_outliers (row %d)" % st.err_index)
+    return out, mask, flags, st

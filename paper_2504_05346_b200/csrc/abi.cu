@@ -17,6 +17,13 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b, float damp_rel, 
                                      float* xnorm, void* workspace, size_t ws_bytes,
                                      int32_t* status_dev, cudaStream_t stream);
 size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
+size_t prune_outliers_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
+thanos_status_t prune_layer_outliers_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+                                          thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                          const float* U, const float* xnorm, const float* H,
+                                          int32_t n, int32_t m, int32_t B, double alpha,
+                                          uint8_t* row_flags_out, void* workspace, size_t ws_bytes,
+                                          thanos_stats_t* stats, cudaStream_t stream);
 thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, double p, int32_t n,
                                     int32_t m, int32_t B);
 thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b, const float* U,
@@ -118,6 +125,29 @@ thanos_status_t thanos_prune_layer(const void* W_in, void* W_out, uint8_t* mask_
   if (!workspace || ws_bytes < prune_workspace_bytes(c, b, B, wdtype)) return THANOS_ERR_WORKSPACE;
   return prune_layer_impl(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, mode, p, n, m, B,
                           workspace, ws_bytes, stats_dev, static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prune_layer_outliers(const void* W_in, void* W_out, uint8_t* mask_out,
+                                            thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                            const float* factor, const float* xnorm,
+                                            const float* H, int32_t n, int32_t m, int32_t B,
+                                            double alpha, uint8_t* row_outlier_out,
+                                            void* workspace, size_t ws_bytes,
+                                            thanos_stats_t* stats_dev, void* stream) {
+  if (!W_in || !W_out || !mask_out || !factor || !xnorm || !H || !stats_dev)
+    return THANOS_ERR_INVALID_ARG;
+  if (!dtype_ok(wdtype)) return THANOS_ERR_DTYPE;
+  if (!(alpha >= 0.0 && alpha < 1.0)) return THANOS_ERR_INVALID_ARG;
+  THANOS_TRY(validate_sweep_args(c, b, THANOS_NM, 0.0, n, m, B));
+  if (c > (1 << 24)) return THANOS_ERR_SHAPE;
+  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(mask_out) || !aligned16(factor) ||
+      !aligned16(xnorm) || !aligned16(H) || !aligned16(workspace) || !aligned16(stats_dev))
+    return THANOS_ERR_ALIGNMENT;
+  if (!workspace || ws_bytes < prune_outliers_workspace_bytes(c, b, B, wdtype))
+    return THANOS_ERR_WORKSPACE;
+  return prune_layer_outliers_impl(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, H, n, m, B,
+                                   alpha, row_outlier_out, workspace, ws_bytes, stats_dev,
+                                   static_cast<cudaStream_t>(stream));
 }
 
 thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t b,
@@ -293,6 +323,9 @@ size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, th
     case THANOS_WS_PRUNE:
       if (c < 1 || B < 1 || B > 512) return 0;
       return prune_workspace_bytes(c, b, B, dtype);
+    case THANOS_WS_PRUNE_OUTLIERS:
+      if (c < 1 || B < 1 || B > 512) return 0;
+      return prune_outliers_workspace_bytes(c, b, B, dtype);
     case THANOS_WS_HOST_LAYER:
       if (c < 1 || B < 1 || B > 512) return 0;
       return host_layout(c, b, B, dtype).total;

@@ -599,11 +599,11 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
 __global__ void __launch_bounds__(256)
 nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
                uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, int n, int m,
-               thanos_stats_t* stats) {
+               thanos_stats_t* stats, const uint8_t* __restrict__ row_skip, int n_skip) {
   const int groups = Bw / m;
   int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (idx == 0) {  // launches of one sweep are ordered, so one thread can keep the books
-    stats->n_pruned += (long long)c * groups * n;
+    stats->n_pruned += (long long)(c - n_skip) * groups * n;
     stats->n_blocks += 1;
   }
   if (idx >= (int64_t)c * groups) return;
@@ -613,6 +613,10 @@ nm_mark_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
   unsigned key[32];
   for (int e = 0; e < m; ++e) key[e] = metric_key(w[e], __ldg(&x[e]));
   uint8_t* mo = mask + (int64_t)row * b + j1 + g * m;
+  if (row_skip && row_skip[row]) {  // outlier row (Algorithm 4's row loop stops before them)
+    for (int e = 0; e < m; ++e) mo[e] = 0;
+    return;
+  }
   for (int e = 0; e < m; ++e) {
     // rank of e = number of entries that come before it in (key, column) order
     int rk = 0;
@@ -648,6 +652,79 @@ __global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long lo
   thanos_stats_t z = {};
   z.r_left = r;
   *stats = z;
+}
+
+// ------------------------------------------------------------------ outlier rows (Algorithm 4)
+// h_i = ||W_i X||^2 = 1/2 W_i H W_i^T from T = W H: one warp per row.
+__global__ void __launch_bounds__(256)
+row_loss_kernel(const float* __restrict__ Wc, const float* __restrict__ Tm, int c, int b,
+                float* __restrict__ h) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= c) return;
+  const float4* w = reinterpret_cast<const float4*>(Wc + (int64_t)row * b);
+  const float4* t = reinterpret_cast<const float4*>(Tm + (int64_t)row * b);
+  double acc = 0.0;
+  for (int q = lane; q < (b >> 2); q += 32) {
+    const float4 a = w[q], v = t[q];
+    acc += (double)a.x * v.x + (double)a.y * v.y + (double)a.z * v.z + (double)a.w * v.w;
+  }
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) h[row] = fmaxf((float)(0.5 * acc), 0.f);
+}
+
+// The n_out rows with the largest h (order (h, row): of equal losses the higher row index is the
+// larger) get flag 1.  One CTA: radix select of the n_out-th largest key, then the ties.
+__global__ void __launch_bounds__(1024)
+outlier_rows_kernel(const float* __restrict__ h, int c, int n_out, uint8_t* __restrict__ flags) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix, s_k, s_gt;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    s_prefix = 0;
+    s_k = (unsigned)n_out;  // rank from the top still to resolve
+  }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const unsigned prefix = s_prefix;
+    for (int i = tid; i < c; i += 1024) {
+      const unsigned key = __float_as_uint(h[i]);
+      if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned k = s_k, bin = 255;
+      for (;; --bin) {  // from the largest digit down
+        if (hist[bin] >= k || bin == 0) break;
+        k -= hist[bin];
+      }
+      s_prefix = (prefix << 8) | bin;
+      s_k = k;
+    }
+    __syncthreads();
+  }
+  const unsigned tau = s_prefix;  // key of the n_out-th largest loss
+  if (tid == 0) s_gt = 0;
+  __syncthreads();
+  unsigned gt = 0;
+  for (int i = tid; i < c; i += 1024) {
+    const unsigned key = __float_as_uint(h[i]);
+    flags[i] = key > tau ? 1 : 0;
+    gt += key > tau;
+  }
+  atomicAdd(&s_gt, gt);
+  __syncthreads();
+  if (tid == 0) {
+    int need = n_out - (int)s_gt;
+    for (int i = c - 1; i >= 0 && need > 0; --i) {
+      if (__float_as_uint(h[i]) == tau) {
+        flags[i] = 1;
+        --need;
+      }
+    }
+  }
 }
 
 struct SweepWs {
@@ -721,7 +798,8 @@ thanos_status_t prepare_blocks(const float* U, int b, int B, const SweepWs& w,
 
 thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* xnorm,
                            thanos_mode_t mode, int n, int m, int B, int j1, int64_t* r_ext,
-                           const SweepWs& w, thanos_stats_t* stats, cudaStream_t stream) {
+                           const SweepWs& w, thanos_stats_t* stats, cudaStream_t stream,
+                           const uint8_t* row_skip = nullptr, int n_skip = 0) {
   const int Bw = (b - j1 < B) ? b - j1 : B;
   const int j2 = j1 + Bw;
   const int bb = j1 / B;
@@ -751,7 +829,7 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     s_fixed = Bw / m * n;
     int64_t items = (int64_t)c * (Bw / m);
     nm_mark_kernel<<<(unsigned)ceil_div(items, 256), 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1,
-                                                                      Bw, n, m, stats);
+                                                                      Bw, n, m, stats, row_skip, n_skip);
     THANOS_CHECK_LAUNCH();
   }
   THANOS_TRY(launch_block_solve(Wc, mask, w.G + (size_t)bb * B * B, w.S + (size_t)bb * B * B, B,
@@ -834,11 +912,33 @@ thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b,
   return THANOS_OK;
 }
 
-thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+namespace {
+
+struct OutlierWs {
+  __nv_bfloat16* Wp;  // [3][c, b] planes of the weights
+  __nv_bfloat16* Hp;  // [3][b, b] planes of the Hessian
+  float* T;           // [c, b] W H
+  float* h;           // [c] row losses
+  uint8_t* flags;     // [c] 1 = outlier row
+};
+
+size_t outlier_extra_bytes(int64_t c, int64_t b) {
+  size_t t = round_up(3 * (size_t)c * b * sizeof(__nv_bfloat16), 256);
+  t += round_up(3 * (size_t)b * b * sizeof(__nv_bfloat16), 256);
+  t += round_up((size_t)c * b * sizeof(float), 256);
+  t += round_up((size_t)c * sizeof(float), 256);
+  t += round_up((size_t)c, 256);
+  return t + 256;
+}
+
+// The whole sweep.  With H and alpha > 0 (n:m mode) the ceil(alpha c) rows with the largest
+// h_i = 1/2 W_i H W_i^T are found first and left untouched (Algorithm 4, outlier rows).
+thanos_status_t prune_layer_core(const void* W_in, void* W_out, uint8_t* mask_out,
                                  thanos_dtype_t wdtype, int64_t c, int64_t b, const float* U,
                                  const float* xnorm, thanos_mode_t mode, double p, int32_t n,
                                  int32_t m, int32_t B, void* workspace, size_t ws_bytes,
-                                 thanos_stats_t* stats, cudaStream_t stream) {
+                                 thanos_stats_t* stats, cudaStream_t stream, const float* H,
+                                 double alpha, uint8_t* row_flags_out) {
   SweepWs w;
   const bool need_wc = wdtype != THANOS_F32;
   if (!carve(w, workspace, ws_bytes, c, b, B, need_wc)) return THANOS_ERR_WORKSPACE;
@@ -855,15 +955,56 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
                                   cudaMemcpyDeviceToDevice, stream));
   }
   THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
+  THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
+  const uint8_t* row_skip = nullptr;
+  int n_skip = 0;
+  if (H != nullptr) {
+    // outlier rows: h = 1/2 rowdot(W, W H), then the ceil(alpha c) largest
+    n_skip = alpha > 0.0 ? (int)ceil(alpha * (double)c - 1e-12) : 0;
+    const size_t base = prune_workspace_bytes(c, b, B, wdtype);
+    if (ws_bytes < base + outlier_extra_bytes(c, b)) return THANOS_ERR_WORKSPACE;
+    Arena ar(static_cast<char*>(workspace) + base, ws_bytes - base);
+    OutlierWs o;
+    o.Wp = ar.take<__nv_bfloat16>(3 * (size_t)nel);
+    o.Hp = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
+    o.T = ar.take<float>((size_t)nel);
+    o.h = ar.take<float>((size_t)c);
+    o.flags = ar.take<uint8_t>((size_t)c);
+    if (!ar.ok()) return THANOS_ERR_WORKSPACE;
+    THANOS_TRY(split3_planes(Wc, b, c, b, o.Wp, b, nel, stream));
+    THANOS_TRY(split3_planes(H, b, b, b, o.Hp, b, b * b, stream));
+    TcGemmArgs g;
+    g.D = o.T;
+    g.ldd = b;
+    g.A = o.Wp;
+    g.lda = b;
+    g.a_plane = nel;
+    g.B = o.Hp;
+    g.ldb = b;
+    g.b_plane = b * b;
+    g.b_kmajor = 0;
+    g.M = (int)c;
+    g.N = (int)b;
+    g.K = (int)b;
+    g.status = w.tc_status;
+    THANOS_TRY(tc_gemm_split3(g, stream));
+    row_loss_kernel<<<(unsigned)ceil_div(c, 8), 256, 0, stream>>>(Wc, o.T, (int)c, (int)b, o.h);
+    THANOS_CHECK_LAUNCH();
+    outlier_rows_kernel<<<1, 1024, 0, stream>>>(o.h, (int)c, n_skip, o.flags);
+    THANOS_CHECK_LAUNCH();
+    if (row_flags_out)
+      THANOS_CUDA(cudaMemcpyAsync(row_flags_out, o.flags, (size_t)c, cudaMemcpyDeviceToDevice,
+                                  stream));
+    row_skip = o.flags;
+  }
   long long r = 0;
   if (mode == THANOS_UNSTRUCTURED) r = (long long)floor(p * (double)c * (double)b);
   init_sweep_kernel<<<1, 1, 0, stream>>>(w.st, stats, r);
   THANOS_CHECK_LAUNCH();
-  THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
   for (int64_t j1 = 0; j1 < b; j1 += B) {
     THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr, w,
-                          stats, stream));
+                          stats, stream, row_skip, n_skip));
   }
   fold_tc_status_kernel<<<1, 1, 0, stream>>>(stats, w.tc_status);
   THANOS_CHECK_LAUNCH();
@@ -872,6 +1013,31 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
     THANOS_CHECK_LAUNCH();
   }
   return THANOS_OK;
+}
+
+}  // namespace
+
+thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+                                 thanos_dtype_t wdtype, int64_t c, int64_t b, const float* U,
+                                 const float* xnorm, thanos_mode_t mode, double p, int32_t n,
+                                 int32_t m, int32_t B, void* workspace, size_t ws_bytes,
+                                 thanos_stats_t* stats, cudaStream_t stream) {
+  return prune_layer_core(W_in, W_out, mask_out, wdtype, c, b, U, xnorm, mode, p, n, m, B,
+                          workspace, ws_bytes, stats, stream, nullptr, 0.0, nullptr);
+}
+
+size_t prune_outliers_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
+  return prune_workspace_bytes(c, b, B, dtype) + outlier_extra_bytes(c, b);
+}
+
+thanos_status_t prune_layer_outliers_impl(const void* W_in, void* W_out, uint8_t* mask_out,
+                                          thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                          const float* U, const float* xnorm, const float* H,
+                                          int32_t n, int32_t m, int32_t B, double alpha,
+                                          uint8_t* row_flags_out, void* workspace, size_t ws_bytes,
+                                          thanos_stats_t* stats, cudaStream_t stream) {
+  return prune_layer_core(W_in, W_out, mask_out, wdtype, c, b, U, xnorm, THANOS_NM, 0.0, n, m, B,
+                          workspace, ws_bytes, stats, stream, H, alpha, row_flags_out);
 }
 
 }  // namespace thanos

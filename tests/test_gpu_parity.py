@@ -438,6 +438,51 @@ def test_argument_errors_are_reported(T):
     assert st.status == 0
 
 
+# ------------------------------------------------------------------------------ outlier rows
+@pytest.mark.parametrize("c,b,dtype,n,m,B,alpha", [
+    (96, 256, "f32", 2, 4, 64, 0.1), (160, 384, "bf16", 2, 4, 128, 0.05),
+    (64, 256, "f32", 4, 8, 64, 0.3), (50, 128, "f32", 2, 4, 32, 0.0)])
+def test_outlier_rows_parity(T, c, b, dtype, n, m, B, alpha):
+    """Algorithm 4 with alpha: outlier flags, untouched outlier rows, and the other rows against
+    the oracle (rows are independent in n:m mode)."""
+    W = WL.make_weight(c, b, dtype, seed=81, layer_index=c)
+    g = torch.Generator().manual_seed(c + b)
+    scale = torch.exp(0.7 * torch.randn((c, 1), generator=g))   # spread the row losses
+    W = (W.float() * scale).to(W.dtype)
+    Xt = WL.make_activations(2048, b, dtype, "student_t4", 0.02, 0, 10.0, 29, 0, mix=0.5)
+    H = _gpu_hessian(T, Xt)
+    H64, W64 = _np64(H), _np64(W)
+    U, xn = T.prepare_inverse(H, 0.01)
+    Wp, M, flags, st = T.prune_layer_outliers(W.to(DEV), U, xn, H, n, m, alpha, B=B)
+    torch.cuda.synchronize()
+    # outlier rows: the ceil(alpha c) largest h_i (differences only between near-equal losses)
+    h = O.row_losses(W64, H=H64)
+    sigma, n_out = O.outlier_row_order(h, alpha)
+    fo = np.zeros(c, dtype=np.uint8)
+    fo[sigma[c - n_out:]] = 1
+    fg = flags.cpu().numpy()
+    assert int(fg.sum()) == n_out
+    if n_out:
+        hb = h[sigma[c - n_out]]                     # smallest outlier loss
+        for i in np.nonzero(fg != fo)[0]:
+            assert abs(h[i] - hb) <= 1e-5 * hb
+    Mg, Wg = M.cpu().numpy(), _np64(Wp)
+    out_rows = fg.astype(bool)
+    assert np.array_equal(Wg[out_rows], W64[out_rows]) and Mg[out_rows].sum() == 0
+    assert st.n_pruned == (c - n_out) * b // m * n == int(Mg.sum())
+    # the pruned rows against the oracle's n:m sweep (alpha does not change them)
+    Wo, Mo, _ = O.thanos_nm(W64, None, n, m, B, 0.01, H=H64, alpha=0.0)
+    rows = ~out_rows & ~(Mg != Mo).any(axis=1)
+    assert rows.sum() >= 0.9 * (c - n_out)
+    Wo_cmp = _np64(torch.tensor(Wo).to(torch.bfloat16)) if dtype == "bf16" else Wo
+    tol = PU.TOL_W_BF16 if dtype == "bf16" else PU.TOL_W_F32
+    assert PU.rel_fro(Wg[rows], Wo_cmp[rows]) <= tol
+    if alpha > 0 and np.array_equal(fg, fo):
+        Wa, Ma, _ = O.thanos_nm(W64, None, n, m, B, 0.01, H=H64, alpha=alpha)
+        assert np.array_equal(Ma[out_rows], Mg[out_rows])
+        assert np.array_equal(Wa[out_rows], W64[out_rows])
+
+
 # ------------------------------------------------------------------------------ bench-size
 def test_full_size_layer_sampled_rows(T):
     """4096 x 4096 bf16 layer, B = 128 (benchmark shape), 50 % unstructured and 2:4: structural
