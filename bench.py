@@ -503,7 +503,11 @@ def run_single_layer(args):
             continue
         U, xn = T.prepare_inverse(H, cfg.damp_rel)
         ev[2].record()
-        _, _, st = T.prune_layer(W, U, xn, B=cfg.B, **margs)
+        if args.alpha >= 0.0:   # n:m with outlier rows (2:4 unless the workload names an n:m)
+            n_, m_ = (cfg.n, cfg.m) if cfg.mode == "nm" else (2, 4)
+            _, _, _, st = T.prune_layer_outliers(W, U, xn, H, n_, m_, args.alpha, B=cfg.B)
+        else:
+            _, _, st = T.prune_layer(W, U, xn, B=cfg.B, **margs)
         ev[3].record()
         torch.cuda.synchronize()
         out.append({"hessian_ms": round(ev[0].elapsed_time(ev[1]), 4),
@@ -531,6 +535,8 @@ def main():
                     help="profile driver: one c x b layer with a tokens instead of the layer set")
     ap.add_argument("--hessian-only", action="store_true", help="with --single-layer: stop after H")
     ap.add_argument("--reps", type=int, default=1)
+    ap.add_argument("--alpha", type=float, default=-1.0,
+                    help="with --single-layer: n:m sweep with this fraction of outlier rows")
     args = ap.parse_args()
     if args.single_layer:
         run_single_layer(args)
