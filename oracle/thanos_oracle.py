@@ -275,6 +275,66 @@ def thanos_nm(W, X, n, m, B, damp_rel=0.0, H=None, collect=None, alpha=0.0):
 
 
 # --------------------------------------------------------------------------------------
+# Structured pruning (Algorithm 2): whole columns, one shared system for all rows
+# --------------------------------------------------------------------------------------
+def column_losses(W_rows, xnorm):
+    """``v_j = ||W_{rows, j} (x) X_j||_F^2 = ||W_{rows, j}||^2 ||X_j||^2`` over the rows that are
+    pruned (Eq. for the column loss, Section 4.7; ``xnorm_j = ||X_j||_2``)."""
+    W_rows = np.asarray(W_rows, dtype=F64)
+    return np.sum(W_rows ** 2, axis=0) * np.asarray(xnorm, dtype=F64) ** 2
+
+
+def structured_column_count(p, b, alpha):
+    """``s = ceil(p b / (1 - alpha))`` columns are removed (Algorithm 2, first line)."""
+    return int(math.ceil(float(p) * b / (1.0 - float(alpha)) - 1e-12))
+
+
+def thanos_structured(W, X, p, alpha=0.0, damp_rel=0.0, H=None):
+    """Algorithm 2.  Rows are permuted so that the ``ceil(alpha c)`` outlier rows (largest
+    ``h_i``) come last, columns so that the ``s`` columns with the smallest ``v_j`` come first;
+    the pruned rows get ``W - W[:, :s] inv(Hinv[:s, :s]) Hinv[:s, :]`` (Eq. 8 with the same ``q``
+    for every row) and exact zeros in the removed columns; the permutations are undone.
+    Outlier rows are not changed at all.  Returns ``(W_pruned, removed_columns, outlier_rows, H)``
+    with boolean index arrays in the original order.
+
+    Readings: the listing writes the update as an assignment to ``W[:, 1:s]`` with a right-hand
+    side of width ``b`` -- taken as the update of the whole (pruned) rows, as in Eq. 8; ``H^{-1}``
+    is the inverse of the damped Hessian; ties in ``v_j`` keep the column order."""
+    W = np.asarray(W, dtype=F64)
+    c, b = W.shape
+    if H is None:
+        H = hessian(X)
+    xn = feature_norms(H)
+    s = structured_column_count(p, b, alpha)
+    if not 0 <= s < b:
+        raise ValueError("p / (1 - alpha) must leave at least one column")
+    if alpha > 0:
+        sigma_r, n_out = outlier_row_order(row_losses(W, H=H), alpha)
+    else:
+        sigma_r, n_out = np.arange(c), 0
+    Wq = W[sigma_r]                                   # W' = Q W
+    n_rows = c - n_out
+    v = column_losses(Wq[:n_rows], xn)
+    sigma_c = np.argsort(v, kind="stable")            # columns with the smallest loss first
+    Wp = Wq[:, sigma_c]                               # W' P
+    Hinv = np.linalg.inv(damped(H, damp_rel))[np.ix_(sigma_c, sigma_c)]
+    if s > 0:
+        lam = np.linalg.solve(Hinv[:s, :s].T, Wp[:n_rows, :s].T).T   # W[:, :s] inv(Hinv[:s,:s])
+        Wp[:n_rows] = Wp[:n_rows] - lam @ Hinv[:s, :]
+        Wp[:n_rows, :s] = 0.0
+    inv_c = np.empty(b, dtype=np.int64)
+    inv_c[sigma_c] = np.arange(b)
+    inv_r = np.empty(c, dtype=np.int64)
+    inv_r[sigma_r] = np.arange(c)
+    out = Wp[:, inv_c][inv_r]
+    removed = np.zeros(b, dtype=bool)
+    removed[sigma_c[:s]] = True
+    outl = np.zeros(c, dtype=bool)
+    outl[sigma_r[n_rows:]] = True
+    return out, removed, outl, H
+
+
+# --------------------------------------------------------------------------------------
 # Faster float64 route for larger shapes: one factorisation instead of one inverse per block.
 # Allowed only because tests show it equals the literal sweep to ~1e-10 on small shapes.
 # --------------------------------------------------------------------------------------

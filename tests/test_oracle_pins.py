@@ -384,3 +384,59 @@ def test_outlier_rows_are_the_largest_losses_and_stay_untouched():
     assert np.array_equal(Mz, M0) and np.array_equal(Wz, W0)
     s2, n2 = O.outlier_row_order(np.array([1.0, 3.0, 3.0, 0.5]), 0.25)
     assert n2 == 1 and list(s2) == [3, 0, 1, 2]    # of the tied rows 1 and 2, row 2 is the outlier
+
+
+# ------------------------------------------------------------------------------ structured
+def test_column_losses_match_the_frobenius_definition():
+    rng = np.random.default_rng(8)
+    W = rng.standard_normal((5, 7))
+    X = rng.standard_normal((7, 30))
+    xn = O.feature_norms(O.hessian(X))
+    v = O.column_losses(W, xn)
+    for j in range(7):
+        outer = np.outer(W[:, j], X[j])             # W_{:, j} (x) X_j
+        assert abs(v[j] - np.linalg.norm(outer, "fro") ** 2) <= 1e-10 * v[j]
+    assert O.structured_column_count(0.3, 10, 0.0) == 3
+    assert O.structured_column_count(0.3, 10, 0.25) == 4     # ceil(3 / 0.75)
+
+
+def test_structured_is_the_constrained_least_squares_refit():
+    """Pruned rows: zeros in the s removed columns, and the kept columns minimise
+    ||(w_hat - w) X'||^2 (X' = X with the damping appended) -- a plain lstsq; outlier rows are
+    returned unchanged; the removed columns are the s smallest v_j."""
+    rng = np.random.default_rng(9)
+    c, b, a = 9, 14, 60
+    W = rng.standard_normal((c, b))
+    X = rng.standard_normal((b, a)) * rng.uniform(0.5, 2.0, size=(b, 1))
+    W[4] *= 25.0
+    for alpha, p in ((0.0, 0.3), (0.1, 0.25)):
+        Wp, removed, outl, H = O.thanos_structured(W, X, p, alpha, damp_rel=0.02)
+        s = O.structured_column_count(p, b, alpha)
+        assert removed.sum() == s
+        n_out = int(math.ceil(alpha * c - 1e-12)) if alpha > 0 else 0
+        assert outl.sum() == n_out and (n_out == 0 or outl[4])
+        assert np.array_equal(Wp[outl], W[outl])
+        rows = ~outl
+        assert np.all(Wp[np.ix_(rows, removed)] == 0.0)
+        v = O.column_losses(W[rows], O.feature_norms(H))
+        assert v[removed].max() <= v[~removed].min()
+        lam = 0.02 * np.mean(np.diag(H))
+        Xd = np.concatenate([X, np.sqrt(lam / 2.0) * np.eye(b)], axis=1)   # 2 Xd Xd^T = H + lam I
+        keep = ~removed
+        for i in np.nonzero(rows)[0]:
+            sol, *_ = np.linalg.lstsq(Xd[keep].T, (W[i] @ Xd), rcond=None)
+            assert np.allclose(Wp[i, keep], sol, rtol=1e-8, atol=1e-10)
+
+
+def test_structured_single_column_is_the_obs_closed_form():
+    rng = np.random.default_rng(10)
+    c, b = 3, 6
+    W = rng.standard_normal((c, b))
+    X = rng.standard_normal((b, 40))
+    Wp, removed, outl, H = O.thanos_structured(W, X, 1.0 / b, 0.0, damp_rel=0.0)
+    q = int(np.nonzero(removed)[0][0])
+    Hinv = np.linalg.inv(H)
+    for i in range(c):
+        want = W[i] - (W[i, q] / Hinv[q, q]) * Hinv[q]      # Eq. 3
+        want[q] = 0.0
+        assert np.allclose(Wp[i], want, rtol=1e-9, atol=1e-12)
