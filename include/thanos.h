@@ -168,6 +168,40 @@ thanos_status_t thanos_prune_layer_outliers(const void* W_in, void* W_out, uint8
                                             thanos_stats_t* stats_dev, void* stream);
 
 /*
+ * Structured pruning (Algorithm 2, Section 4.7): whole columns are removed.  With
+ * s = ceil(p b / (1 - alpha)), the ceil(alpha c) rows with the largest h_i (as in
+ * thanos_prune_layer_outliers) are left untouched; over the other rows the s columns with the
+ * smallest v_j = ||W_{rows, j}||_2^2 ||X_j||_2^2 form q (equal losses: the lower column first), and
+ * every pruned row gets the multi-weight update of Eq. 8 with this same q,
+ *     W <- W - W[:, q] inv(Hinv[q, q]) Hinv[q, :],   W[:, q] <- 0   (Hinv = inverse damped Hessian).
+ * The listing permutes columns and rows to bring q and the pruned rows first and undoes both at
+ * the end; this call gathers by index instead, which is the same arithmetic.
+ *
+ *  W_in, W_out   device [c, b] of wdtype, row-major, may alias.
+ *  col_removed_out  device uint8 [b] or NULL: 1 for the removed columns.
+ *  row_outlier_out  device uint8 [c] or NULL: 1 for the outlier rows.
+ *  factor, xnorm    from thanos_prepare_inverse.
+ *  H        device fp32 [b, b], the undamped Hessian; may be NULL when alpha == 0.
+ *  p        0 <= p < 1, alpha 0 <= alpha < 1, and s < b, else THANOS_ERR_INVALID_ARG.
+ *  b % 8 == 0, 8 <= b <= 65536, 1 <= c <= 2^24.
+ *  stats_dev  device thanos_stats_t, written by this call: n_pruned = s (c - ceil(alpha c)),
+ *           max_s = s, status THANOS_ERR_NOT_SPD if Hinv[q, q] is not positive definite in fp32.
+ *  workspace: thanos_structured_workspace_bytes(c, b, p, alpha, wdtype) bytes.
+ * Asynchronous on stream; no allocation.
+ */
+thanos_status_t thanos_prune_layer_structured(const void* W_in, void* W_out,
+                                              uint8_t* col_removed_out, uint8_t* row_outlier_out,
+                                              thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                              const float* factor, const float* xnorm,
+                                              const float* H, double p, double alpha,
+                                              void* workspace, size_t ws_bytes,
+                                              thanos_stats_t* stats_dev, void* stream);
+
+/* Workspace of thanos_prune_layer_structured; 0 if the arguments are not accepted. */
+size_t thanos_structured_workspace_bytes(int64_t c, int64_t b, double p, double alpha,
+                                         thanos_dtype_t dtype);
+
+/*
  * One block step of the sweep from a caller-supplied state (the body of the block loop of
  * Algorithm 1 / Algorithm 4), for step-by-step checking against a reference.
  *

@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     prune_layer_noalloc,
     dense_product,
     prune_layer_outliers,
+    prune_layer_structured,
     workspace_bytes,
     launch_count,
     status_string,

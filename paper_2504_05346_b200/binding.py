@@ -88,6 +88,12 @@ def load_library():
     lib.thanos_prune_layer_outliers.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp, i32, i32, i32,
                                                 ctypes.c_double, vp, vp, sz, vp, vp]
     lib.thanos_prune_layer_outliers.restype = i32
+    lib.thanos_prune_layer_structured.argtypes = [vp, vp, vp, vp, i32, i64, i64, vp, vp, vp,
+                                                  ctypes.c_double, ctypes.c_double, vp, sz, vp, vp]
+    lib.thanos_prune_layer_structured.restype = i32
+    lib.thanos_structured_workspace_bytes.argtypes = [i64, i64, ctypes.c_double, ctypes.c_double,
+                                                      i32]
+    lib.thanos_structured_workspace_bytes.restype = sz
     lib.thanos_prune_block.argtypes = [vp, vp, i64, i64, vp, vp, i32, i32, i32, i32, i64, vp, vp,
                                        sz, vp, vp]
     lib.thanos_prune_block.restype = i32
@@ -372,3 +378,41 @@ def prune_layer_outliers(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Ten
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_outliers (row %d)" % st.err_index)
     return out, mask, flags, st
+
+
+def prune_layer_structured(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tensor, p: float,
+                           alpha: float = 0.0, H: Optional[torch.Tensor] = None, stream=None,
+                           workspace: Optional[torch.Tensor] = None,
+                           out: Optional[torch.Tensor] = None):
+    """thanos_prune_layer_structured: removes the ceil(p b / (1 - alpha)) columns of smallest loss
+    from all but the ceil(alpha c) outlier rows and updates the kept weights (Algorithm 2).
+    Returns (W_pruned, removed columns uint8 [b], outlier rows uint8 [c], stats)."""
+    lib = load_library()
+    _check_dev(W, factor, xnorm)
+    if alpha > 0.0:
+        if H is None:
+            raise ValueError("alpha > 0 needs the Hessian H")
+        _check_dev(H)
+    c, b = W.shape
+    dt = _dtype_code(W)
+    if out is None:
+        out = torch.empty_like(W)
+    colrm = torch.empty((b,), dtype=torch.uint8, device=W.device)
+    flags = torch.empty((c,), dtype=torch.uint8, device=W.device)
+    stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
+    if workspace is None:
+        need = int(lib.thanos_structured_workspace_bytes(c, b, float(p), float(alpha), dt))
+        if need == 0:
+            raise ThanosError(1, "thanos_structured_workspace_bytes rejected the arguments")
+        workspace = _ws(need, W.device)
+    _check(lib.thanos_prune_layer_structured(W.data_ptr(), out.data_ptr(), colrm.data_ptr(),
+                                             flags.data_ptr(), dt, c, b, factor.data_ptr(),
+                                             xnorm.data_ptr(),
+                                             H.data_ptr() if H is not None else None, float(p),
+                                             float(alpha), workspace.data_ptr(), workspace.numel(),
+                                             stats.data_ptr(), _stream_ptr(stream)),
+           "thanos_prune_layer_structured")
+    st = _read_stats(stats)
+    if st.status != 0:
+        raise ThanosError(st.status, "thanos_prune_layer_structured (index %d)" % st.err_index)
+    return out, colrm, flags, st

@@ -24,6 +24,14 @@ thanos_status_t prune_layer_outliers_impl(const void* W_in, void* W_out, uint8_t
                                           int32_t n, int32_t m, int32_t B, double alpha,
                                           uint8_t* row_flags_out, void* workspace, size_t ws_bytes,
                                           thanos_stats_t* stats, cudaStream_t stream);
+size_t structured_workspace_bytes(int64_t c, int64_t b, double p, double alpha,
+                                  thanos_dtype_t dtype);
+thanos_status_t prune_layer_structured_impl(const void* W_in, void* W_out, uint8_t* col_removed_out,
+                                            uint8_t* row_outlier_out, thanos_dtype_t wdtype,
+                                            int64_t c, int64_t b, const float* U,
+                                            const float* xnorm, const float* H, double p,
+                                            double alpha, void* workspace, size_t ws_bytes,
+                                            thanos_stats_t* stats, cudaStream_t stream);
 thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, double p, int32_t n,
                                     int32_t m, int32_t B);
 thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b, const float* U,
@@ -148,6 +156,36 @@ thanos_status_t thanos_prune_layer_outliers(const void* W_in, void* W_out, uint8
   return prune_layer_outliers_impl(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, H, n, m, B,
                                    alpha, row_outlier_out, workspace, ws_bytes, stats_dev,
                                    static_cast<cudaStream_t>(stream));
+}
+
+thanos_status_t thanos_prune_layer_structured(const void* W_in, void* W_out,
+                                              uint8_t* col_removed_out, uint8_t* row_outlier_out,
+                                              thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                              const float* factor, const float* xnorm,
+                                              const float* H, double p, double alpha,
+                                              void* workspace, size_t ws_bytes,
+                                              thanos_stats_t* stats_dev, void* stream) {
+  if (!W_in || !W_out || !factor || !xnorm || !stats_dev) return THANOS_ERR_INVALID_ARG;
+  if (!dtype_ok(wdtype)) return THANOS_ERR_DTYPE;
+  if (!(alpha >= 0.0 && alpha < 1.0) || !(p >= 0.0 && p < 1.0)) return THANOS_ERR_INVALID_ARG;
+  if (alpha > 0.0 && !H) return THANOS_ERR_INVALID_ARG;
+  if (c < 1 || c > (1 << 24) || b < 8 || b > MAX_B || b % 8 != 0) return THANOS_ERR_SHAPE;
+  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(factor) || !aligned16(xnorm) ||
+      !aligned16(H) || !aligned16(workspace) || !aligned16(stats_dev))
+    return THANOS_ERR_ALIGNMENT;
+  const size_t need = structured_workspace_bytes(c, b, p, alpha, wdtype);
+  if (need == 0) return THANOS_ERR_INVALID_ARG;  // p / (1 - alpha) leaves no column
+  if (!workspace || ws_bytes < need) return THANOS_ERR_WORKSPACE;
+  return prune_layer_structured_impl(W_in, W_out, col_removed_out, row_outlier_out, wdtype, c, b,
+                                     factor, xnorm, H, p, alpha, workspace, ws_bytes, stats_dev,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+size_t thanos_structured_workspace_bytes(int64_t c, int64_t b, double p, double alpha,
+                                         thanos_dtype_t dtype) {
+  if (c < 1 || b < 8 || b > MAX_B || b % 8 != 0 || !dtype_ok(dtype)) return 0;
+  if (!(alpha >= 0.0 && alpha < 1.0) || !(p >= 0.0 && p < 1.0)) return 0;
+  return structured_workspace_bytes(c, b, p, alpha, dtype);
 }
 
 thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t b,

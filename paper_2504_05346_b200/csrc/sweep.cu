@@ -922,6 +922,8 @@ struct OutlierWs {
   uint8_t* flags;     // [c] 1 = outlier row
 };
 
+}  // namespace
+
 size_t outlier_extra_bytes(int64_t c, int64_t b) {
   size_t t = round_up(3 * (size_t)c * b * sizeof(__nv_bfloat16), 256);
   t += round_up(3 * (size_t)b * b * sizeof(__nv_bfloat16), 256);
@@ -930,6 +932,47 @@ size_t outlier_extra_bytes(int64_t c, int64_t b) {
   t += round_up((size_t)c, 256);
   return t + 256;
 }
+
+// Outlier rows (Algorithms 2 and 4): h = 1/2 rowdot(W, W H), then flag 1 on the n_out rows with
+// the largest h.  scratch holds outlier_extra_bytes(c, b); *flags_dev points into it.
+thanos_status_t outlier_row_flags(const float* Wc, const float* H, int64_t c, int64_t b, int n_out,
+                                  void* scratch, size_t scratch_bytes, uint8_t** flags_dev,
+                                  int32_t* tc_status, cudaStream_t stream) {
+  const int64_t nel = c * b;
+  Arena ar(scratch, scratch_bytes);
+  OutlierWs o;
+  o.Wp = ar.take<__nv_bfloat16>(3 * (size_t)nel);
+  o.Hp = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
+  o.T = ar.take<float>((size_t)nel);
+  o.h = ar.take<float>((size_t)c);
+  o.flags = ar.take<uint8_t>((size_t)c);
+  if (!ar.ok()) return THANOS_ERR_WORKSPACE;
+  THANOS_TRY(split3_planes(Wc, b, c, b, o.Wp, b, nel, stream));
+  THANOS_TRY(split3_planes(H, b, b, b, o.Hp, b, b * b, stream));
+  TcGemmArgs g;
+  g.D = o.T;
+  g.ldd = b;
+  g.A = o.Wp;
+  g.lda = b;
+  g.a_plane = nel;
+  g.B = o.Hp;
+  g.ldb = b;
+  g.b_plane = b * b;
+  g.b_kmajor = 0;
+  g.M = (int)c;
+  g.N = (int)b;
+  g.K = (int)b;
+  g.status = tc_status;
+  THANOS_TRY(tc_gemm_split3(g, stream));
+  row_loss_kernel<<<(unsigned)ceil_div(c, 8), 256, 0, stream>>>(Wc, o.T, (int)c, (int)b, o.h);
+  THANOS_CHECK_LAUNCH();
+  outlier_rows_kernel<<<1, 1024, 0, stream>>>(o.h, (int)c, n_out, o.flags);
+  THANOS_CHECK_LAUNCH();
+  *flags_dev = o.flags;
+  return THANOS_OK;
+}
+
+namespace {
 
 // The whole sweep.  With H and alpha > 0 (n:m mode) the ceil(alpha c) rows with the largest
 // h_i = 1/2 W_i H W_i^T are found first and left untouched (Algorithm 4, outlier rows).
@@ -963,39 +1006,13 @@ thanos_status_t prune_layer_core(const void* W_in, void* W_out, uint8_t* mask_ou
     n_skip = alpha > 0.0 ? (int)ceil(alpha * (double)c - 1e-12) : 0;
     const size_t base = prune_workspace_bytes(c, b, B, wdtype);
     if (ws_bytes < base + outlier_extra_bytes(c, b)) return THANOS_ERR_WORKSPACE;
-    Arena ar(static_cast<char*>(workspace) + base, ws_bytes - base);
-    OutlierWs o;
-    o.Wp = ar.take<__nv_bfloat16>(3 * (size_t)nel);
-    o.Hp = ar.take<__nv_bfloat16>(3 * (size_t)b * b);
-    o.T = ar.take<float>((size_t)nel);
-    o.h = ar.take<float>((size_t)c);
-    o.flags = ar.take<uint8_t>((size_t)c);
-    if (!ar.ok()) return THANOS_ERR_WORKSPACE;
-    THANOS_TRY(split3_planes(Wc, b, c, b, o.Wp, b, nel, stream));
-    THANOS_TRY(split3_planes(H, b, b, b, o.Hp, b, b * b, stream));
-    TcGemmArgs g;
-    g.D = o.T;
-    g.ldd = b;
-    g.A = o.Wp;
-    g.lda = b;
-    g.a_plane = nel;
-    g.B = o.Hp;
-    g.ldb = b;
-    g.b_plane = b * b;
-    g.b_kmajor = 0;
-    g.M = (int)c;
-    g.N = (int)b;
-    g.K = (int)b;
-    g.status = w.tc_status;
-    THANOS_TRY(tc_gemm_split3(g, stream));
-    row_loss_kernel<<<(unsigned)ceil_div(c, 8), 256, 0, stream>>>(Wc, o.T, (int)c, (int)b, o.h);
-    THANOS_CHECK_LAUNCH();
-    outlier_rows_kernel<<<1, 1024, 0, stream>>>(o.h, (int)c, n_skip, o.flags);
-    THANOS_CHECK_LAUNCH();
+    uint8_t* flags = nullptr;
+    THANOS_TRY(outlier_row_flags(Wc, H, c, b, n_skip, static_cast<char*>(workspace) + base,
+                                 ws_bytes - base, &flags, w.tc_status, stream));
     if (row_flags_out)
-      THANOS_CUDA(cudaMemcpyAsync(row_flags_out, o.flags, (size_t)c, cudaMemcpyDeviceToDevice,
+      THANOS_CUDA(cudaMemcpyAsync(row_flags_out, flags, (size_t)c, cudaMemcpyDeviceToDevice,
                                   stream));
-    row_skip = o.flags;
+    row_skip = flags;
   }
   long long r = 0;
   if (mode == THANOS_UNSTRUCTURED) r = (long long)floor(p * (double)c * (double)b);

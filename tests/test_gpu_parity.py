@@ -588,3 +588,39 @@ def test_dense_product_matches_float64(T, M, N, K, bt):
     got2 = _np64(big[:, :N])
     assert np.max(np.abs(got2 - (_np64(C0) - 0.5 * want)) / (scale + np.abs(_np64(C0)))) <= 3e-6
     assert float(big[:, N:].abs().max()) == 0.0
+
+
+# ------------------------------------------------------------------------------ structured
+@pytest.mark.parametrize("c,b,dtype,p,alpha", [
+    (96, 256, "f32", 0.3, 0.0), (200, 384, "f32", 0.25, 0.1), (160, 512, "bf16", 0.5, 0.05),
+    (64, 136, "f32", 0.1, 0.0), (40, 128, "f32", 0.0, 0.0), (300, 1032, "f32", 0.4, 0.02)])
+def test_structured_parity(T, c, b, dtype, p, alpha):
+    """Algorithm 2: removed columns, outlier rows and the updated weights against the oracle."""
+    W = WL.make_weight(c, b, dtype, seed=91, layer_index=c)
+    g = torch.Generator().manual_seed(c + b)
+    W = (W.float() * torch.exp(0.7 * torch.randn((c, 1), generator=g))
+         * torch.exp(0.5 * torch.randn((1, b), generator=g))).to(W.dtype)
+    Xt = WL.make_activations(max(2048, 3 * b), b, dtype, "student_t4", 0.02, 0, 10.0, 31, 0, mix=0.5)
+    H = _gpu_hessian(T, Xt)
+    H64, W64 = _np64(H), _np64(W)
+    U, xn = T.prepare_inverse(H, 0.01)
+    Wp, colrm, flags, st = T.prune_layer_structured(W.to(DEV), U, xn, p, alpha,
+                                                    H=H if alpha > 0 else None)
+    torch.cuda.synchronize()
+    Wo, rm_o, out_o, _ = O.thanos_structured(W64, None, p, alpha, 0.01, H=H64)
+    s = O.structured_column_count(p, b, alpha)
+    rm_g, out_g = colrm.cpu().numpy().astype(bool), flags.cpu().numpy().astype(bool)
+    assert rm_g.sum() == s == st.max_s and out_g.sum() == out_o.sum()
+    assert st.n_pruned == s * (c - int(out_o.sum()))
+    assert np.array_equal(out_g, out_o), "outlier rows differ"
+    assert np.array_equal(rm_g, rm_o), "removed columns differ"
+    Wg = _np64(Wp)
+    assert np.array_equal(Wg[out_g], W64[out_g])                  # outlier rows untouched
+    assert np.all(Wg[np.ix_(~out_g, rm_g)] == 0.0)                # exact zeros
+    Wo_cmp = _np64(torch.tensor(Wo).to(torch.bfloat16)) if dtype == "bf16" else Wo
+    tol = PU.TOL_W_BF16 if dtype == "bf16" else PU.TOL_W_F32
+    assert PU.rel_fro(Wg, Wo_cmp) <= tol
+    if dtype == "f32" and s:
+        # the change of the kept weights itself, not hidden behind the unchanged mass of W
+        d_g, d_o = Wg - W64, Wo - W64
+        assert PU.rel_fro(d_g[:, ~rm_g], d_o[:, ~rm_g]) <= 2e-4
