@@ -503,7 +503,11 @@ def run_single_layer(args):
             continue
         U, xn = T.prepare_inverse(H, cfg.damp_rel)
         ev[2].record()
-        if args.alpha >= 0.0:   # n:m with outlier rows (2:4 unless the workload names an n:m)
+        if args.structured > 0.0:   # Algorithm 2: whole columns, with --alpha outlier rows
+            al = max(args.alpha, 0.0)
+            _, _, _, st = T.prune_layer_structured(W, U, xn, args.structured, al,
+                                                   H=H if al > 0 else None)
+        elif args.alpha >= 0.0:   # n:m with outlier rows (2:4 unless the workload names an n:m)
             n_, m_ = (cfg.n, cfg.m) if cfg.mode == "nm" else (2, 4)
             _, _, _, st = T.prune_layer_outliers(W, U, xn, H, n_, m_, args.alpha, B=cfg.B)
         else:
@@ -537,6 +541,8 @@ def main():
     ap.add_argument("--reps", type=int, default=1)
     ap.add_argument("--alpha", type=float, default=-1.0,
                     help="with --single-layer: n:m sweep with this fraction of outlier rows")
+    ap.add_argument("--structured", type=float, default=0.0, metavar="P",
+                    help="with --single-layer: structured pruning of this fraction of the columns")
     args = ap.parse_args()
     if args.single_layer:
         run_single_layer(args)

@@ -334,6 +334,21 @@ def thanos_structured(W, X, p, alpha=0.0, damp_rel=0.0, H=None):
     return out, removed, outl, H
 
 
+def structured_update_rows(W_rows, removed, Hd):
+    """Eq. 8 for given rows with a given set of removed columns ``q`` (boolean [b]):
+    ``w - w_q inv(Hinv[q, q]) Hinv[q, :]`` and zeros at ``q`` -- the row update of Algorithm 2
+    without its permutations, for checking sampled rows of a large layer."""
+    W_rows = np.asarray(W_rows, dtype=F64)
+    q = np.nonzero(np.asarray(removed, dtype=bool))[0]
+    if q.size == 0:
+        return W_rows.copy()
+    Hinv = np.linalg.inv(np.asarray(Hd, dtype=F64))
+    lam = np.linalg.solve(Hinv[np.ix_(q, q)].T, W_rows[:, q].T).T
+    out = W_rows - lam @ Hinv[q, :]
+    out[:, q] = 0.0
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # Faster float64 route for larger shapes: one factorisation instead of one inverse per block.
 # Allowed only because tests show it equals the literal sweep to ~1e-10 on small shapes.

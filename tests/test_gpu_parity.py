@@ -624,3 +624,40 @@ def test_structured_parity(T, c, b, dtype, p, alpha):
         # the change of the kept weights itself, not hidden behind the unchanged mass of W
         d_g, d_o = Wg - W64, Wo - W64
         assert PU.rel_fro(d_g[:, ~rm_g], d_o[:, ~rm_g]) <= 2e-4
+
+
+def test_structured_full_size_sampled_rows(T):
+    """4096 x 4096 bf16 layer, 30 % of the columns with 10 % outlier rows: the removed columns are
+    the smallest losses of the oracle, and sampled rows match Eq. 8 in float64 for that set."""
+    c = b = 4096
+    p, alpha = 0.3, 0.1
+    W = WL.make_weight(c, b, "bf16", seed=2, layer_index=0, device=DEV)
+    Xd = WL.make_activations(16384, b, "bf16", "student_t4", 0.005, 0, 50.0, 2, 0, device=DEV)
+    H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(H, Xd)
+    U, xn = T.prepare_inverse(H, 0.01)
+    Wp, colrm, flags, st = T.prune_layer_structured(W, U, xn, p, alpha, H=H)
+    torch.cuda.synchronize()
+    H64, W64 = _np64(H), _np64(W)
+    s = O.structured_column_count(p, b, alpha)
+    rm, outl = colrm.cpu().numpy().astype(bool), flags.cpu().numpy().astype(bool)
+    n_out = int(np.ceil(alpha * c - 1e-12))
+    assert rm.sum() == s and outl.sum() == n_out and st.n_pruned == s * (c - n_out)
+    h = O.row_losses(W64, H=H64)
+    sigma, _ = O.outlier_row_order(h, alpha)
+    hb = h[sigma[c - n_out]]
+    fo = np.zeros(c, dtype=bool)
+    fo[sigma[c - n_out:]] = True
+    for i in np.nonzero(fo != outl)[0]:
+        assert abs(h[i] - hb) <= 1e-5 * hb
+    v = O.column_losses(W64[~outl], O.feature_norms(H64))
+    vs = np.sort(v)
+    lo, hi = vs[s - 1], vs[s]
+    assert v[rm].max() <= hi * (1 + 1e-6) and v[~rm].min() >= lo * (1 - 1e-6)
+    Wg = _np64(Wp)
+    assert np.array_equal(Wg[outl], W64[outl])
+    assert bool((Wp[:, colrm.bool()][~flags.bool()] == 0).all())
+    rows = np.nonzero(~outl)[0][[0, 1, 1000, 2500, -1]]
+    Wr = O.structured_update_rows(W64[rows], rm, O.damped(H64, 0.01))
+    Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
+    assert PU.rel_fro(Wg[rows], Wr) <= PU.TOL_W_BF16

@@ -440,3 +440,12 @@ def test_structured_single_column_is_the_obs_closed_form():
         want = W[i] - (W[i, q] / Hinv[q, q]) * Hinv[q]      # Eq. 3
         want[q] = 0.0
         assert np.allclose(Wp[i], want, rtol=1e-9, atol=1e-12)
+
+
+def test_structured_update_rows_agrees_with_algorithm_2():
+    rng = np.random.default_rng(11)
+    W = rng.standard_normal((6, 12))
+    X = rng.standard_normal((12, 50))
+    Wp, removed, outl, H = O.thanos_structured(W, X, 0.25, 0.0, damp_rel=0.01)
+    rows = O.structured_update_rows(W[[1, 4]], removed, O.damped(H, 0.01))
+    assert np.allclose(rows, Wp[[1, 4]], rtol=1e-10, atol=1e-12)
