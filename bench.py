@@ -12,6 +12,7 @@ sample of the same workload instead.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -482,6 +483,8 @@ def run_single_layer(args):
     T.load_library()
     c, b, a = [int(v) for v in args.single_layer.split(",")]
     cfg = WL.CONFIGS[args.workload]
+    if args.block > 0:
+        cfg = dataclasses.replace(cfg, B=args.block)
     dev = torch.device("cuda", 0)
     margs = mode_args(cfg, T)
     W = WL.make_weight(c, b, cfg.dtype, seed=cfg.seed, layer_index=0, device=dev)
@@ -541,6 +544,8 @@ def main():
     ap.add_argument("--reps", type=int, default=1)
     ap.add_argument("--alpha", type=float, default=-1.0,
                     help="with --single-layer: n:m sweep with this fraction of outlier rows")
+    ap.add_argument("--block", type=int, default=0,
+                    help="with --single-layer: block width B instead of the workload's")
     ap.add_argument("--structured", type=float, default=0.0, metavar="P",
                     help="with --single-layer: structured pruning of this fraction of the columns")
     args = ap.parse_args()

@@ -133,8 +133,8 @@ thanos_status_t thanos_prepare_inverse(const float* H, int64_t b, float damp_rel
  *  mode UNSTRUCTURED: 0 <= p < 1 (n, m ignored).  Metric ties are broken by (row, column)
  *  ascending.  mode NM: 0 < n < m <= 32, B % m == 0, b % m == 0; n weights are REMOVED per
  *  group; ties by column ascending.
- *  1 <= B <= 512, B % 8 == 0, b % 8 == 0.  Per-row systems up to s = 320 unknowns are
- *  supported (s <= B; s = n B / m in NM mode); larger -> THANOS_ERR_SHAPE.
+ *  1 <= B <= 512, B % 8 == 0, b % 8 == 0.  A row solves a system of min(|q|, |k|) <= B / 2
+ *  unknowns (direct or complement form), so every admissible B is supported in both modes.
  *  stats_dev device thanos_stats_t, zeroed by this call.
  *  workspace: thanos_workspace_bytes(THANOS_WS_PRUNE, c, b, B, wdtype) bytes.
  */

@@ -420,124 +420,7 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   }
 }
 
-// General kernel for systems too large for the fast one: one warp per row, packed lower
-// triangle in shared memory, column-by-column Cholesky, direct form only.
-__global__ void __launch_bounds__(256)
-solve_rows_general_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
-                          const float* __restrict__ G, int ldg, __nv_bfloat16* __restrict__ D,
-                          int64_t dplane, int c, int b, int j1, int Bw, int ldd, int smax,
-                          int report_max_s,
-                          thanos_stats_t* stats) {
-  extern __shared__ __align__(16) unsigned char dyn[];
-  const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-  const int warps = blockDim.x >> 5;
-  const size_t tri = (size_t)smax * (smax + 1) / 2;
-  const size_t per_warp = ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
-  float* L = reinterpret_cast<float*>(dyn + per_warp * warp);
-  float* y = L + tri;
-  short* q = reinterpret_cast<short*>(y + smax);
-
-  for (int row = blockIdx.x * warps + warp; row < c; row += gridDim.x * warps) {
-    const uint8_t* mrow = mask + (int64_t)row * b + j1;
-    float* wrow = Wc + (int64_t)row * b + j1;
-    int s = 0;
-    for (int base = 0; base < Bw; base += 32) {
-      int jj = base + lane;
-      bool mb = jj < Bw && mrow[jj] != 0;
-      unsigned bal = __ballot_sync(FULL, mb);
-      if (mb) {
-        int pos = s + __popc(bal & ((1u << lane) - 1u));
-        if (pos < smax) q[pos] = (short)jj;
-      }
-      s += __popc(bal);
-    }
-    if (s > smax) {  // cannot happen for a valid mask; refuse rather than overrun
-      if (lane == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
-      s = 0;
-    }
-    __syncwarp();
-    if (s == 0) {
-      for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
-      continue;
-    }
-    if (report_max_s && row == 0 && lane == 0) atomicMax(&stats->max_s, s);
-    for (int a = 0; a < s; ++a) {
-      const float* Grow = G + (int64_t)q[a] * ldg;
-      float* Lrow = L + (size_t)a * (a + 1) / 2;
-      for (int bb = lane; bb <= a; bb += 32) Lrow[bb] = Grow[q[bb]];
-    }
-    for (int a = lane; a < s; a += 32) y[a] = wrow[q[a]];
-    __syncwarp();
-    bool bad = false;
-    for (int j = 0; j < s; ++j) {
-      float* Lj = L + (size_t)j * (j + 1) / 2;
-      float part = 0.f;
-      for (int k = lane; k < j; k += 32) part = fmaf(Lj[k], Lj[k], part);
-      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(FULL, part, o);
-      float d = Lj[j] - part;
-      if (!(d > 0.f) || !isfinite(d)) {
-        bad = true;
-        d = 1.f;
-      }
-      float ljj = sqrtf(d);
-      float inv = 1.f / ljj;
-      __syncwarp();
-      if (lane == 0) Lj[j] = ljj;
-      for (int i = j + 1 + lane; i < s; i += 32) {
-        float* Li = L + (size_t)i * (i + 1) / 2;
-        float v = Li[j];
-        for (int k = 0; k < j; ++k) v = fmaf(-Li[k], Lj[k], v);
-        Li[j] = v * inv;
-      }
-      __syncwarp();
-    }
-    if (bad) {
-      if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
-      for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
-      continue;
-    }
-    for (int j = 0; j < s; ++j) {
-      float zj = y[j] / L[(size_t)j * (j + 1) / 2 + j];
-      __syncwarp();
-      if (lane == 0) y[j] = zj;
-      for (int i = j + 1 + lane; i < s; i += 32)
-        y[i] = fmaf(-L[(size_t)i * (i + 1) / 2 + j], zj, y[i]);
-      __syncwarp();
-    }
-    for (int j = s - 1; j >= 0; --j) {
-      const float* Lj = L + (size_t)j * (j + 1) / 2;
-      float xj = y[j] / Lj[j];
-      __syncwarp();
-      if (lane == 0) y[j] = xj;
-      for (int k = lane; k < j; k += 32) y[k] = fmaf(-Lj[k], xj, y[k]);
-      __syncwarp();
-    }
-    // delta = -lambda-hat G[q, :] on the kept columns, -w on the removed ones
-    for (int jj = lane; jj < Bw; jj += 32) {
-      const float w = wrow[jj];
-      float d;
-      if (mrow[jj] != 0) {
-        d = -w;
-        wrow[jj] = 0.f;
-      } else {
-        float g = 0.f;
-        for (int a = 0; a < s; ++a) g = fmaf(y[a], G[(int64_t)q[a] * ldg + jj], g);
-        d = -g;
-        wrow[jj] = w + d;
-      }
-      store_split3(D + (int64_t)row * ldd + jj, dplane, d);
-    }
-    __syncwarp();
-  }
-}
-
 constexpr size_t SOLVE_SMEM_BUDGET = 227 * 1024;  // the most dynamic shared memory a CTA can get
-
-size_t general_per_warp_bytes(int smax) {
-  size_t tri = (size_t)smax * (smax + 1) / 2;
-  return ((tri + smax) * sizeof(float) + smax * sizeof(short) + 15) / 16 * 16;
-}
 
 template <int NR>
 thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, const float* S,
@@ -567,10 +450,18 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
 
 }  // namespace
 
-// Largest system the general kernel can hold for one warp.
+int cta_solve_max_unknowns();
+thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                 int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
+                                 int Bw, int ldd, int n_max, const int* row_lists,
+                                 const unsigned* list_counts, int fixed_kind, int report_max_s,
+                                 thanos_stats_t* stats, cudaStream_t stream);
+
+// Systems of up to 159 unknowns go to the warp-per-row kernel, larger ones to the CTA-per-row
+// kernel; n_small_max is the largest min(|q|, |k|) a row can have.
 bool solve_supported(int s_direct_max, int n_small_max) {
-  if (n_small_max + 1 <= 160) return true;
-  return general_per_warp_bytes(s_direct_max) <= SOLVE_SMEM_BUDGET;
+  (void)s_direct_max;
+  return n_small_max <= cta_solve_max_unknowns();
 }
 
 // Solves every row of the block [j1, j1 + Bw): writes the block's new weights into Wc and the
@@ -584,28 +475,13 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
                                    thanos_stats_t* stats, cudaStream_t stream) {
   const bool uniform = s_fixed >= 0;
   const int n_small = uniform ? (s_fixed < Bw - s_fixed ? s_fixed : Bw - s_fixed) : Bw / 2;
-  if (n_small + 1 > 160) {
-    const int smax = uniform ? s_fixed : Bw;
-    size_t per_warp = general_per_warp_bytes(smax < 1 ? 1 : smax);
-    int warps = (int)(SOLVE_SMEM_BUDGET / per_warp);
-    if (warps < 1) return THANOS_ERR_SHAPE;
-    if (warps > 8) warps = 8;
-    {
-    static std::atomic<unsigned long long> done{0};
-    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_general_kernel, (int)SOLVE_SMEM_BUDGET, done));
-  }
-    int64_t grid = ceil_div(c, warps);
-    if (grid > 148 * 4) grid = 148 * 4;
-    solve_rows_general_kernel<<<(unsigned)grid, warps * 32, per_warp * warps, stream>>>(
-        Wc, mask, G, ld_mat, D, dplane, c, b, j1, Bw, ldd, smax < 1 ? 1 : smax, uniform ? 1 : 0,
-        stats);
-    THANOS_CHECK_LAUNCH();
-    return THANOS_OK;
-  }
   const int fixed_kind = uniform ? (s_fixed > Bw - s_fixed ? 1 : 0) : 0;
   const int* rl = uniform ? nullptr : row_lists;
   const unsigned* lc = uniform ? nullptr : list_counts;
   const int rep = uniform ? 1 : 0;
+  if (n_small + 1 > 160)
+    return launch_cta_solve(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
+                            fixed_kind, rep, stats, stream);
   if (n_small + 1 <= 32)
     return launch_fast<1>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                           fixed_kind, rep, stats, stream);

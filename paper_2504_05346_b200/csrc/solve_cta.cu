@@ -1,0 +1,439 @@
+// Per-row constrained solve for large systems (Eqs. 5-8): one CTA per row.
+//
+// Same mathematics as the warp-per-row kernel (direct form on G for rows with |q| <= |k|,
+// complement form on S otherwise), for systems of 160 to 319 unknowns -- e.g. 2:4 sparsity with
+// the block width B = 512 of Section 5, where every row solves a 256 x 256 system.  The gathered
+// matrix lives in shared memory as the lower triangle of 16 x 16 tiles (1 KB each, 16-byte chunks
+// swizzled by the row so that the accesses below are free of bank conflicts); the right-hand
+// side is appended as row n, so that the factorisation L L^T also yields y = L^{-1} rhs.
+// Right-looking tile Cholesky by 8 warps: panel solve (one thread per row), trailing update
+// (one warp per target tile, handed out by a shared counter); warp 0 updates and factors the
+// next diagonal tile first, which takes the only serial step off the critical path.  Blocked
+// back substitution L^T x = y, then the change of the block's weights as in the small kernel.
+#include "common.cuh"
+
+namespace thanos {
+
+namespace {
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int CTA_THREADS = 256;
+constexpr int CTA_WARPS = CTA_THREADS / 32;
+constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 - 1 = 319 unknowns
+
+__device__ __forceinline__ void put_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
+#pragma unroll
+  for (int pl = 0; pl < 3; ++pl) {
+    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
+    p[(int64_t)pl * plane] = hb;
+    d -= __bfloat162float(hb);
+  }
+}
+
+// tile (I, J), J <= I, of the lower triangle; 256 floats each
+__device__ __forceinline__ int tile_base(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
+// 16-byte chunk c of row r sits at chunk position c ^ ((r >> 1) & 3)
+__device__ __forceinline__ int chunk_off(int r, int c) { return (r << 4) + (((c ^ (r >> 1)) & 3) << 2); }
+__device__ __forceinline__ int elem_off(int r, int k) { return chunk_off(r, k >> 2) + (k & 3); }
+
+__host__ __device__ inline size_t cta_smem_bytes(int tiles, int Bw) {
+  // tiles, invd / xs / rhs [16 tiles + 16 each], wblk / dvec [Bw], two index lists, scan scratch
+  const size_t fl = (size_t)(tiles * (tiles + 1) / 2) * 256 + 3 * (16 * (size_t)tiles + 16) + 2 * (size_t)Bw;
+  return fl * 4 + 2 * 2 * (size_t)(Bw + 16) + 64;
+}
+
+// Cholesky of the diagonal tile (K, K) by one warp: lane r < 16 holds row r.  Columns >= n (the
+// right-hand-side row and the identity padding) get pivot 1.
+__device__ __forceinline__ bool factor_diag_tile(float* __restrict__ Tt, float* __restrict__ invd,
+                                                 int col0, int n, int lane) {
+  const int r = lane & 15;
+  float a[16];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float4 v = *reinterpret_cast<const float4*>(Tt + chunk_off(r, c));
+    a[4 * c] = v.x; a[4 * c + 1] = v.y; a[4 * c + 2] = v.z; a[4 * c + 3] = v.w;
+  }
+  bool bad = false;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    float dj = __shfl_sync(FULL, a[j], j);
+    if (col0 + j < n) {
+      if (!(dj > 0.f) || !isfinite(dj)) {
+        bad = true;
+        dj = 1.f;
+      }
+    } else {
+      dj = 1.f;
+    }
+    const float rinv = rsqrtf(dj);
+    if (lane == 0) invd[col0 + j] = rinv;
+    a[j] *= rinv;
+#pragma unroll
+    for (int v = j + 1; v < 16; ++v) {
+      const float lvj = __shfl_sync(FULL, a[j], v);
+      a[v] = fmaf(-a[j], lvj, a[v]);
+    }
+  }
+  if (lane < 16) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      *reinterpret_cast<float4*>(Tt + chunk_off(r, c)) =
+          make_float4(a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
+  }
+  __syncwarp();
+  return bad;
+}
+
+// C -= A B^T for 16 x 16 tiles by one warp: lane (lr, lc) owns rows lr, lr + 8 and columns
+// lc, lc + 4, lc + 8, lc + 12.
+__device__ __forceinline__ void tile_update(float* __restrict__ Ct, const float* __restrict__ At,
+                                            const float* __restrict__ Bt, int lane) {
+  const int lr = lane >> 2, lc = lane & 3;
+  float acc[2][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) acc[0][i] = acc[1][i] = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float4 a0 = *reinterpret_cast<const float4*>(At + chunk_off(lr, c));
+    const float4 a1 = *reinterpret_cast<const float4*>(At + chunk_off(lr + 8, c));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 bv = *reinterpret_cast<const float4*>(Bt + chunk_off(lc + 4 * i, c));
+      acc[0][i] = fmaf(a0.x, bv.x, acc[0][i]);
+      acc[0][i] = fmaf(a0.y, bv.y, acc[0][i]);
+      acc[0][i] = fmaf(a0.z, bv.z, acc[0][i]);
+      acc[0][i] = fmaf(a0.w, bv.w, acc[0][i]);
+      acc[1][i] = fmaf(a1.x, bv.x, acc[1][i]);
+      acc[1][i] = fmaf(a1.y, bv.y, acc[1][i]);
+      acc[1][i] = fmaf(a1.z, bv.z, acc[1][i]);
+      acc[1][i] = fmaf(a1.w, bv.w, acc[1][i]);
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int r = lr + 8 * h;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float* p = Ct + chunk_off(r, i) + lc;  // column lc + 4 i: chunk i, element lc
+      *p -= acc[h][i];
+    }
+  }
+}
+
+// exclusive prefix sum of one value per thread over the CTA (256 threads)
+__device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* warp_sums,
+                                                       unsigned& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  unsigned incl = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned y = __shfl_up_sync(FULL, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();
+  if (lane == 31) warp_sums[wid] = incl;
+  __syncthreads();
+  unsigned before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < CTA_WARPS; ++w) {
+    const unsigned v = warp_sums[w];
+    if (w < wid) before += v;
+    all += v;
+  }
+  total = all;
+  return before + incl - x;
+}
+
+// Rows come from row_lists[2][c] / list_counts[2] (kind 0: |q| <= |k|, direct form on G; kind 1:
+// complement form on S), or are all rows with kind `fixed_kind` when row_lists is null.
+__global__ void __launch_bounds__(CTA_THREADS, 1)
+solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
+                      const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
+                      __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
+                      int ldd, int tiles, const int* __restrict__ row_lists,
+                      const unsigned* __restrict__ list_counts, int fixed_kind, int report_max_s,
+                      thanos_stats_t* stats) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  float* A = reinterpret_cast<float*>(dyn);
+  float* invd = A + (size_t)(tiles * (tiles + 1) / 2) * 256;
+  float* xs = invd + 16 * tiles + 16;
+  float* rhsv = xs + 16 * tiles + 16;
+  float* wblk = rhsv + 16 * tiles + 16;
+  float* dvec = wblk + Bw;
+  unsigned short* qlist = reinterpret_cast<unsigned short*>(dvec + Bw);
+  unsigned short* klist = qlist + Bw + 16;
+  unsigned* scratch = reinterpret_cast<unsigned*>(klist + Bw + 16);  // 16 words
+  unsigned* warp_sums = scratch;          // [8]
+  unsigned* s_counter = scratch + 9;
+  unsigned* s_bad = scratch + 10;
+
+  int cnt0, cnt1;
+  if (row_lists) {
+    cnt0 = (int)list_counts[0];
+    cnt1 = (int)list_counts[1];
+  } else {
+    cnt0 = fixed_kind == 0 ? c : 0;
+    cnt1 = fixed_kind == 0 ? 0 : c;
+  }
+  for (int li = blockIdx.x; li < cnt0 + cnt1; li += gridDim.x) {
+    const bool kpath = li >= cnt0;
+    const int row = row_lists ? (kpath ? row_lists[(size_t)c + (li - cnt0)] : row_lists[li]) : li;
+    const float* __restrict__ M = kpath ? Sm : Gm;
+    const uint8_t* mrow = mask + (int64_t)row * b + j1;
+    float* wrow = Wc + (int64_t)row * b + j1;
+    __syncthreads();  // the previous row's shared data is no longer read
+    // ---- q = phi(mask row) and its complement k, both ascending: thread t owns columns 2t, 2t+1
+    int s, t;
+    {
+      const int c0 = 2 * tid, c1 = 2 * tid + 1;
+      const int m0 = c0 < Bw ? (int)mrow[c0] : 2, m1 = c1 < Bw ? (int)mrow[c1] : 2;
+      if (c0 < Bw) wblk[c0] = wrow[c0];
+      if (c1 < Bw) wblk[c1] = wrow[c1];
+      const unsigned mine = (unsigned)((m0 == 1) + (m1 == 1)) | ((unsigned)((m0 == 0) + (m1 == 0)) << 16);
+      unsigned all;
+      const unsigned before = cta_exclusive_scan(mine, warp_sums, all);
+      int pq = (int)(before & 0xffffu), pk = (int)(before >> 16);
+      if (m0 == 1) qlist[pq++] = (unsigned short)c0;
+      if (m0 == 0) klist[pk++] = (unsigned short)c0;
+      if (m1 == 1) qlist[pq] = (unsigned short)c1;
+      if (m1 == 0) klist[pk] = (unsigned short)c1;
+      s = (int)(all & 0xffffu);
+      t = (int)(all >> 16);
+    }
+    if (tid == 0) *s_bad = 0;
+    if (s == 0) {  // nothing removed: the row is not touched in this block (CTA-uniform)
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      continue;
+    }
+    if (report_max_s && row == 0 && tid == 0) atomicMax(&stats->max_s, s);
+    const int n = kpath ? t : s;   // unknowns of this row's system
+    const int no = kpath ? s : t;  // size of the other set
+    unsigned short* sel = kpath ? klist : qlist;
+    unsigned short* oth = kpath ? qlist : klist;
+    if (tid < 16) {
+      sel[n + tid] = 0;
+      oth[no + tid] = 0;
+    }
+    const int T = (n + 16) >> 4;   // tile rows of the system plus the right-hand-side row
+    const int Tf = (n + 15) >> 4;  // tile columns that are factored
+    if ((s > t) != kpath || T > tiles) {
+      // cannot happen for lists and launch sizes made by this library
+      if (tid == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      continue;
+    }
+    __syncthreads();
+    // ---- right-hand side: w_q (direct form) or g_e = sum_a w[q_a] S[q_a, k_e] (complement)
+    for (int e = tid; e < n; e += CTA_THREADS) {
+      float g;
+      if (!kpath) {
+        g = wblk[sel[e]];
+      } else {
+        const int col = (int)sel[e];
+        float g0 = 0.f, g1 = 0.f;
+        for (int a = 0; a < no; a += 4) {
+          const ushort4 ix = *reinterpret_cast<const ushort4*>(oth + a);
+          const float w0 = wblk[ix.x];
+          const float w1 = (a + 1 < no) ? wblk[ix.y] : 0.f;
+          const float w2 = (a + 2 < no) ? wblk[ix.z] : 0.f;
+          const float w3 = (a + 3 < no) ? wblk[ix.w] : 0.f;
+          g0 = fmaf(w0, __ldg(M + (int)ix.x * ld_mat + col), g0);
+          g1 = fmaf(w1, __ldg(M + (int)ix.y * ld_mat + col), g1);
+          g0 = fmaf(w2, __ldg(M + (int)ix.z * ld_mat + col), g0);
+          g1 = fmaf(w3, __ldg(M + (int)ix.w * ld_mat + col), g1);
+        }
+        g = g0 + g1;
+      }
+      rhsv[e] = g;
+    }
+    __syncthreads();
+    // ---- gather the lower triangle of M[sel, sel], the right-hand-side row n, identity padding
+    {
+      const int r = tid >> 4, k = tid & 15;
+      const int ntiles = (T * (T + 1)) >> 1;
+      int I = 0, J = 0;
+#pragma unroll 8
+      for (int tt = 0; tt < ntiles; ++tt) {
+        const int i = 16 * I + r, j = 16 * J + k;
+        float v;
+        if (i < n)
+          v = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
+        else if (i == n)
+          v = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
+        else
+          v = i == j ? 1.f : 0.f;
+        A[(tt << 8) + elem_off(r, k)] = v;
+        if (++J > I) {
+          ++I;
+          J = 0;
+        }
+      }
+    }
+    __syncthreads();
+    bool bad = false;
+    if (warp == 0) bad = factor_diag_tile(A + tile_base(0, 0), invd, 0, n, lane);
+    __syncthreads();
+    // ---- right-looking tile Cholesky
+    for (int K = 0; K < Tf; ++K) {
+      const int m = T - K - 1;  // tile rows below the diagonal tile
+      if (tid == 0) *s_counter = 1;
+      // panel: X L_KK^T = A_IK for the rows below, one thread per row
+      {
+        const float* Lk = A + tile_base(K, K);
+        for (int ii = tid; ii < 16 * m; ii += CTA_THREADS) {
+          const int I = K + 1 + (ii >> 4), r = ii & 15;
+          float* arow = A + tile_base(I, K);
+          float x[16];
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            const float4 v = *reinterpret_cast<const float4*>(arow + chunk_off(r, cc));
+            x[4 * cc] = v.x; x[4 * cc + 1] = v.y; x[4 * cc + 2] = v.z; x[4 * cc + 3] = v.w;
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            float l[16];
+#pragma unroll
+            for (int cc = 0; cc <= ((j - 1) >> 2) && j > 0; ++cc) {
+              const float4 v = *reinterpret_cast<const float4*>(Lk + chunk_off(j, cc));
+              l[4 * cc] = v.x; l[4 * cc + 1] = v.y; l[4 * cc + 2] = v.z; l[4 * cc + 3] = v.w;
+            }
+            float acc = x[j];
+#pragma unroll
+            for (int mm = 0; mm < j; ++mm) acc = fmaf(-x[mm], l[mm], acc);
+            x[j] = acc * invd[16 * K + j];
+          }
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc)
+            *reinterpret_cast<float4*>(arow + chunk_off(r, cc)) =
+                make_float4(x[4 * cc], x[4 * cc + 1], x[4 * cc + 2], x[4 * cc + 3]);
+        }
+      }
+      __syncthreads();
+      // trailing update; warp 0 first brings the next diagonal tile up to date and factors it
+      if (warp == 0 && K + 1 < Tf) {
+        float* Ct = A + tile_base(K + 1, K + 1);
+        const float* At = A + tile_base(K + 1, K);
+        tile_update(Ct, At, At, lane);
+        __syncwarp();
+        bad |= factor_diag_tile(Ct, invd, 16 * (K + 1), n, lane);
+      }
+      {
+        // targets (I', J') of the m x m lower triangle in row-major order, index 0 (the next
+        // diagonal tile) excluded; the last one is excluded too when its column is not factored
+        const int total = ((m * (m + 1)) >> 1) - (T > Tf ? 1 : 0);
+        for (;;) {
+          unsigned u = 0;
+          if (lane == 0) u = atomicAdd(s_counter, 1u);
+          u = __shfl_sync(FULL, u, 0);
+          if ((int)u >= total) break;
+          int Ip = (int)((sqrtf(8.f * (float)u + 1.f) - 1.f) * 0.5f);
+          while (((Ip + 1) * (Ip + 2) >> 1) <= (int)u) ++Ip;
+          while (((Ip * (Ip + 1)) >> 1) > (int)u) --Ip;
+          const int Jp = (int)u - ((Ip * (Ip + 1)) >> 1);
+          const int I = K + 1 + Ip, J = K + 1 + Jp;
+          tile_update(A + tile_base(I, J), A + tile_base(I, K), A + tile_base(J, K), lane);
+        }
+      }
+      __syncthreads();
+    }
+    if (warp == 0 && bad && lane == 0) *s_bad = 1;
+    // ---- y = row n of L; blocked back substitution L^T x = y from the bottom
+    {
+      const int In = n >> 4, rn = n & 15;
+      for (int i = tid; i < 16 * T + 4; i += CTA_THREADS)
+        xs[i] = i < n ? A[tile_base(In, i >> 4) + elem_off(rn, i & 15)] : 0.f;
+    }
+    __syncthreads();
+    if (*s_bad) {
+      if (tid == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      continue;
+    }
+    for (int Kb = Tf - 1; Kb >= 0; --Kb) {
+      if (warp == 0) {
+        const float* Lk = A + tile_base(Kb, Kb);
+        const int me = 16 * Kb + (lane & 15);
+        float res = me < n ? xs[me] : 0.f;
+#pragma unroll
+        for (int w = 15; w >= 0; --w) {
+          const int idx = 16 * Kb + w;
+          float xi = __shfl_sync(FULL, res, w);
+          xi = idx < n ? xi * invd[idx] : 0.f;
+          const float lwk = Lk[elem_off(w, lane & 15)];
+          if ((lane & 15) < w) res = fmaf(-lwk, xi, res);
+          if ((lane & 15) == w) res = xi;
+        }
+        if (lane < 16 && me < n) xs[me] = res;
+      }
+      __syncthreads();
+      for (int k = tid; k < 16 * Kb; k += CTA_THREADS) {
+        const float* Lt = A + tile_base(Kb, k >> 4);
+        const int kk = k & 15;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < 16; ++w) acc = fmaf(Lt[elem_off(w, kk)], xs[16 * Kb + w], acc);
+        xs[k] -= acc;
+      }
+      __syncthreads();
+    }
+    // ---- delta over the block
+    for (int a = tid; a < s; a += CTA_THREADS) dvec[qlist[a]] = -wblk[qlist[a]];
+    __syncthreads();
+    if (kpath) {
+      for (int e = tid; e < n; e += CTA_THREADS) dvec[sel[e]] = xs[e];
+    } else {
+      // delta_k = -sum_a lambda_a G[q_a, k_e]
+      for (int e = tid; e < no; e += CTA_THREADS) {
+        const int col = (int)oth[e];
+        float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;
+        for (int a = 0; a < n; a += 4) {
+          const ushort4 ix = *reinterpret_cast<const ushort4*>(sel + a);
+          const float4 xv = *reinterpret_cast<const float4*>(xs + a);
+          g0 = fmaf(xv.x, __ldg(M + (int)ix.x * ld_mat + col), g0);
+          g1 = fmaf(xv.y, __ldg(M + (int)ix.y * ld_mat + col), g1);
+          g2 = fmaf(xv.z, __ldg(M + (int)ix.z * ld_mat + col), g2);
+          g3 = fmaf(xv.w, __ldg(M + (int)ix.w * ld_mat + col), g3);
+        }
+        dvec[col] = -((g0 + g1) + (g2 + g3));
+      }
+    }
+    __syncthreads();
+    for (int jj = tid; jj < Bw; jj += CTA_THREADS) {
+      const float d = dvec[jj];
+      const bool removed = mrow[jj] != 0;
+      wrow[jj] = removed ? 0.f : wblk[jj] + d;
+      put_split3(D + (int64_t)row * ldd + jj, dplane, d);
+    }
+  }
+}
+
+}  // namespace
+
+// Largest system (unknowns) the CTA-per-row kernel holds.
+int cta_solve_max_unknowns() { return 16 * MAX_TILES - 1; }
+
+thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                 int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
+                                 int Bw, int ldd, int n_max, const int* row_lists,
+                                 const unsigned* list_counts, int fixed_kind, int report_max_s,
+                                 thanos_stats_t* stats, cudaStream_t stream) {
+  const int tiles = (n_max + 16) / 16;
+  if (tiles > MAX_TILES || Bw > 2 * CTA_THREADS) return THANOS_ERR_SHAPE;
+  const size_t smem = cta_smem_bytes(tiles, Bw);
+  if (smem > 227 * 1024) return THANOS_ERR_SHAPE;
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_cta_kernel, 227 * 1024, done));
+  }
+  int grid = c < 148 ? c : 148;
+  solve_rows_cta_kernel<<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
+      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,
+      fixed_kind, report_max_s, stats);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+}  // namespace thanos

@@ -261,6 +261,10 @@ SWEEP_CASES = [
     ("wide_block_unstr", 64, 512, 4096, "f32", "student_t4", "unstructured", 0.5, 0, 0, 256, 0.3),
     ("b512_2of4", 48, 1024, 4096, "f32", "student_t4", "nm", 0.0, 2, 4, 512, 0.3),
     ("small_block", 40, 64, 512, "f32", "normal", "unstructured", 0.5, 0, 0, 8, 0.5),
+    ("b512_unstr", 300, 1024, 4096, "f32", "student_t4", "unstructured", 0.5, 0, 0, 512, 0.3),
+    ("b512_unstr70", 160, 1024, 4096, "bf16", "student_t4", "unstructured", 0.7, 0, 0, 512, 0.3),
+    ("b400_unstr", 90, 1200, 4096, "f32", "normal", "unstructured", 0.45, 0, 0, 400, 0.5),
+    ("b512_4of8", 200, 512, 4096, "bf16", "student_t4", "nm", 0.0, 4, 8, 512, 0.0),
 ]
 
 
