@@ -77,33 +77,97 @@ __device__ __forceinline__ unsigned metric_key(float w, float xn) {
 }
 
 // ------------------------------------------------------------------ per-block matrices
-// One CTA per block: dense copy of U_bb (zeros below the diagonal) and V_bb = inv(U_bb) by back
-// substitution, one column of V_bb per thread, accumulated in double.
-__global__ void __launch_bounds__(512)
+// Dense copy of U_bb (zeros below the diagonal) and V_bb = inv(U_bb).  Grid (strips of 64
+// columns, blocks): a CTA owns 64 columns of V_bb and solves U_bb V = I for them by blocked back
+// substitution over row blocks of 32 from the bottom: the finished rows of its strip stay in
+// shared memory, the product with the U tiles to their right and the 32 x 32 triangular solve
+// are accumulated in double.
+constexpr int INV_STRIP = 64;
+constexpr int INV_RB = 32;
+
+__host__ __device__ inline size_t block_inverse_smem(int B) {
+  const size_t rows = (size_t)(B + INV_RB - 1) / INV_RB * INV_RB;
+  return rows * INV_STRIP * sizeof(float) + INV_RB * INV_STRIP * sizeof(double) +
+         INV_RB * (INV_RB + 1) * sizeof(float);
+}
+
+__global__ void __launch_bounds__(256)
 block_inverse_kernel(const float* __restrict__ U, float* __restrict__ Ubb, float* __restrict__ Vbb,
                      int b, int B) {
-  const int bb = blockIdx.x;
+  extern __shared__ __align__(16) unsigned char inv_dyn[];
+  double* Rs = reinterpret_cast<double*>(inv_dyn);                       // [32][64]
+  float* Vs = reinterpret_cast<float*>(Rs + INV_RB * INV_STRIP);         // [B rounded up to 32][64]
+  float* Ut = Vs + (size_t)((B + INV_RB - 1) / INV_RB * INV_RB) * INV_STRIP;  // [32][33]
+  const int tid = threadIdx.x;
+  const int bb = blockIdx.y;
+  const int c0 = blockIdx.x * INV_STRIP;
   const int j1 = bb * B;
   const int Bw = (b - j1 < B) ? b - j1 : B;
   float* Uo = Ubb + (size_t)bb * B * B;
   float* Vo = Vbb + (size_t)bb * B * B;
-  for (int e = threadIdx.x; e < B * B; e += blockDim.x) {
-    const int i = e / B, j = e - i * B;
+  const float* Ub = U + (int64_t)j1 * b + j1;
+  for (int e = tid; e < B * INV_STRIP; e += 256) {
+    const int i = e / INV_STRIP, j = c0 + (e % INV_STRIP);
+    if (j >= B) continue;
     float u = 0.f;
-    if (i < Bw && j < Bw && j >= i) u = U[(int64_t)(j1 + i) * b + j1 + j];
-    Uo[e] = u;
-    Vo[e] = 0.f;
+    if (i < Bw && j < Bw && j >= i) u = Ub[(int64_t)i * b + j];
+    Uo[(size_t)i * B + j] = u;
+  }
+  const int rows_tot = (c0 + INV_STRIP < Bw) ? c0 + INV_STRIP : Bw;  // rows that can be non-zero
+  const int nI = rows_tot > 0 && c0 < Bw ? (rows_tot + INV_RB - 1) / INV_RB : 0;
+  const int col = tid & (INV_STRIP - 1), rg = tid >> 6;  // rows rg, rg + 4, ... of a row block
+  for (int I = nI - 1; I >= 0; --I) {
+    const int r0 = I * INV_RB;
+    double acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+    for (int K = I + 1; K < nI; ++K) {
+      __syncthreads();
+      for (int e = tid; e < INV_RB * INV_RB; e += 256) {
+        const int r = e >> 5, kk = e & 31;
+        const int gi = r0 + r, gk = K * INV_RB + kk;
+        Ut[r * (INV_RB + 1) + kk] = (gi < Bw && gk < Bw) ? Ub[(int64_t)gi * b + gk] : 0.f;
+      }
+      __syncthreads();
+#pragma unroll 4
+      for (int kk = 0; kk < INV_RB; ++kk) {
+        const double v = (double)Vs[(size_t)(K * INV_RB + kk) * INV_STRIP + col];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          acc[i] = fma((double)Ut[(rg + 4 * i) * (INV_RB + 1) + kk], v, acc[i]);
+      }
+    }
+    __syncthreads();
+    for (int e = tid; e < INV_RB * INV_RB; e += 256) {
+      const int r = e >> 5, kk = e & 31;
+      const int gi = r0 + r, gk = r0 + kk;
+      Ut[r * (INV_RB + 1) + kk] = (gi < Bw && gk < Bw && gk >= gi) ? Ub[(int64_t)gi * b + gk] : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = rg + 4 * i;
+      Rs[r * INV_STRIP + col] = ((r0 + r == c0 + col) ? 1.0 : 0.0) - acc[i];
+    }
+    __syncthreads();
+    if (tid < INV_STRIP) {
+      for (int r = INV_RB - 1; r >= 0; --r) {
+        double x = 0.0;
+        if (r0 + r < rows_tot) {
+          x = Rs[r * INV_STRIP + col];
+          for (int k = r + 1; k < INV_RB; ++k)
+            x = fma(-(double)Ut[r * (INV_RB + 1) + k], Rs[k * INV_STRIP + col], x);
+          x /= (double)Ut[r * (INV_RB + 1) + r];
+        }
+        Rs[r * INV_STRIP + col] = x;
+        Vs[(size_t)(r0 + r) * INV_STRIP + col] = (float)x;
+      }
+    }
   }
   __syncthreads();
-  for (int j = threadIdx.x; j < Bw; j += blockDim.x) {
-    // column j of V: U_bb v = e_j, from row j upwards
-    Vo[(size_t)j * B + j] = 1.f / Uo[(size_t)j * B + j];
-    for (int i = j - 1; i >= 0; --i) {
-      double acc = 0.0;
-      for (int k = i + 1; k <= j; ++k)
-        acc += (double)Uo[(size_t)i * B + k] * (double)Vo[(size_t)k * B + j];
-      Vo[(size_t)i * B + j] = (float)(-acc / (double)Uo[(size_t)i * B + i]);
-    }
+  for (int e = tid; e < B * INV_STRIP; e += 256) {
+    const int i = e / INV_STRIP, jj = e % INV_STRIP;
+    if (c0 + jj >= B) continue;
+    Vo[(size_t)i * B + c0 + jj] = (i < nI * INV_RB && i < B) ? Vs[(size_t)i * INV_STRIP + jj] : 0.f;
   }
 }
 
@@ -781,7 +845,12 @@ bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, i
 thanos_status_t prepare_blocks(const float* U, int b, int B, const SweepWs& w,
                                cudaStream_t stream) {
   const int blocks = (int)ceil_div(b, B);
-  block_inverse_kernel<<<blocks, B < 128 ? 128 : B, 0, stream>>>(U, w.Ubb, w.Vbb, b, B);
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(block_inverse_kernel, (int)block_inverse_smem(512), done));
+  }
+  block_inverse_kernel<<<dim3((unsigned)ceil_div(B, INV_STRIP), (unsigned)blocks), 256,
+                         block_inverse_smem(B), stream>>>(U, w.Ubb, w.Vbb, b, B);
   THANOS_CHECK_LAUNCH();
   dim3 gg((unsigned)ceil_div(B, 64), (unsigned)ceil_div(B, 64), (unsigned)blocks);
   block_gram_kernel<0><<<gg, 256, 0, stream>>>(w.Ubb, w.G, b, B);
