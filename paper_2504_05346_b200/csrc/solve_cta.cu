@@ -120,6 +120,69 @@ __device__ __forceinline__ void tile_update(float* __restrict__ Ct, const float*
   }
 }
 
+// 2 x 2 target tiles (I0 + di, J0 + dj) of step K at once: C_IJ -= L_IK L_JK^T.  Lane (lr, lc)
+// owns rows lr, lr + 8 and columns lc + 4 i of every tile, so the operand rows it loads serve
+// four tiles.  Bit 2 di + dj of vmask says that the tile is written; tile indices past the last
+// tile row are clamped for the loads.
+__device__ __forceinline__ void macro_update(float* __restrict__ A, int K, int I0, int J0, int T,
+                                             unsigned vmask, int lane) {
+  const int lr = lane >> 2, lc = lane & 3;
+  const int I1 = I0 + 1 < T ? I0 + 1 : T - 1, J1 = J0 + 1 < T ? J0 + 1 : T - 1;
+  const float* At[2] = {A + tile_base(I0, K), A + tile_base(I1, K)};
+  const float* Bt[2] = {A + tile_base(J0, K), A + tile_base(J1, K)};
+  float acc[2][2][2][4];
+#pragma unroll
+  for (int di = 0; di < 2; ++di)
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int dj = 0; dj < 2; ++dj)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[di][h][dj][i] = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    float4 a[2][2], bv[2][4];
+#pragma unroll
+    for (int di = 0; di < 2; ++di)
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+        a[di][h] = *reinterpret_cast<const float4*>(At[di] + chunk_off(lr + 8 * h, c));
+#pragma unroll
+    for (int dj = 0; dj < 2; ++dj)
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        bv[dj][i] = *reinterpret_cast<const float4*>(Bt[dj] + chunk_off(lc + 4 * i, c));
+#pragma unroll
+    for (int di = 0; di < 2; ++di)
+#pragma unroll
+      for (int dj = 0; dj < 2; ++dj) {
+        if (!(vmask & (1u << (2 * di + dj)))) continue;  // warp-uniform
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float v = acc[di][h][dj][i];
+            v = fmaf(a[di][h].x, bv[dj][i].x, v);
+            v = fmaf(a[di][h].y, bv[dj][i].y, v);
+            v = fmaf(a[di][h].z, bv[dj][i].z, v);
+            v = fmaf(a[di][h].w, bv[dj][i].w, v);
+            acc[di][h][dj][i] = v;
+          }
+      }
+  }
+#pragma unroll
+  for (int di = 0; di < 2; ++di)
+#pragma unroll
+    for (int dj = 0; dj < 2; ++dj) {
+      if (!(vmask & (1u << (2 * di + dj)))) continue;
+      float* Ct = A + tile_base(I0 + di, J0 + dj);
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) Ct[chunk_off(lr + 8 * h, i) + lc] -= acc[di][h][dj][i];
+    }
+}
+
 // exclusive prefix sum of one value per thread over the CTA (256 threads)
 __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* warp_sums,
                                                        unsigned& total) {
@@ -255,21 +318,29 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       const int r = tid >> 4, k = tid & 15;
       const int ntiles = (T * (T + 1)) >> 1;
       int I = 0, J = 0;
-#pragma unroll 8
-      for (int tt = 0; tt < ntiles; ++tt) {
-        const int i = 16 * I + r, j = 16 * J + k;
-        float v;
-        if (i < n)
-          v = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
-        else if (i == n)
-          v = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
-        else
-          v = i == j ? 1.f : 0.f;
-        A[(tt << 8) + elem_off(r, k)] = v;
-        if (++J > I) {
-          ++I;
-          J = 0;
+      for (int t0 = 0; t0 < ntiles; t0 += 8) {  // eight loads in flight per thread
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = 16 * I + r, j = 16 * J + k;
+          float x;
+          if (t0 + u >= ntiles)
+            x = 0.f;
+          else if (i < n)
+            x = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
+          else if (i == n)
+            x = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
+          else
+            x = i == j ? 1.f : 0.f;
+          v[u] = x;
+          if (++J > I) {
+            ++I;
+            J = 0;
+          }
         }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (t0 + u < ntiles) A[((t0 + u) << 8) + elem_off(r, k)] = v[u];
       }
     }
     __syncthreads();
@@ -279,7 +350,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     // ---- right-looking tile Cholesky
     for (int K = 0; K < Tf; ++K) {
       const int m = T - K - 1;  // tile rows below the diagonal tile
-      if (tid == 0) *s_counter = 1;
+      if (tid == 0) *s_counter = 0;
       // panel: X L_KK^T = A_IK for the rows below, one thread per row
       {
         const float* Lk = A + tile_base(K, K);
@@ -321,9 +392,11 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         bad |= factor_diag_tile(Ct, invd, 16 * (K + 1), n, lane);
       }
       {
-        // targets (I', J') of the m x m lower triangle in row-major order, index 0 (the next
-        // diagonal tile) excluded; the last one is excluded too when its column is not factored
-        const int total = ((m * (m + 1)) >> 1) - (T > Tf ? 1 : 0);
+        // the m x m lower triangle of targets in 2 x 2 groups (I', J') in row-major order,
+        // handed out by the shared counter; the next diagonal tile (done by warp 0 above) and a
+        // last column that is not factored are masked out
+        const int m2 = (m + 1) >> 1;
+        const int total = (m2 * (m2 + 1)) >> 1;
         for (;;) {
           unsigned u = 0;
           if (lane == 0) u = atomicAdd(s_counter, 1u);
@@ -333,8 +406,16 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           while (((Ip + 1) * (Ip + 2) >> 1) <= (int)u) ++Ip;
           while (((Ip * (Ip + 1)) >> 1) > (int)u) --Ip;
           const int Jp = (int)u - ((Ip * (Ip + 1)) >> 1);
-          const int I = K + 1 + Ip, J = K + 1 + Jp;
-          tile_update(A + tile_base(I, J), A + tile_base(I, K), A + tile_base(J, K), lane);
+          const int I0 = K + 1 + 2 * Ip, J0 = K + 1 + 2 * Jp;
+          unsigned vmask = 0;
+#pragma unroll
+          for (int di = 0; di < 2; ++di)
+#pragma unroll
+            for (int dj = 0; dj < 2; ++dj) {
+              const int I = I0 + di, J = J0 + dj;
+              if (I < T && J <= I && J < Tf && !(I == K + 1 && J == K + 1)) vmask |= 1u << (2 * di + dj);
+            }
+          if (vmask) macro_update(A, K, I0, J0, T, vmask, lane);
         }
       }
       __syncthreads();
