@@ -17,7 +17,7 @@ namespace thanos {
 namespace {
 
 constexpr unsigned FULL = 0xffffffffu;
-constexpr int CTA_THREADS = 256;
+constexpr int CTA_THREADS = 512;
 constexpr int CTA_WARPS = CTA_THREADS / 32;
 constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 - 1 = 319 unknowns
 
@@ -39,7 +39,7 @@ __device__ __forceinline__ int elem_off(int r, int k) { return chunk_off(r, k >>
 __host__ __device__ inline size_t cta_smem_bytes(int tiles, int Bw) {
   // tiles, invd / xs / rhs [16 tiles + 16 each], wblk / dvec [Bw], two index lists, scan scratch
   const size_t fl = (size_t)(tiles * (tiles + 1) / 2) * 256 + 3 * (16 * (size_t)tiles + 16) + 2 * (size_t)Bw;
-  return fl * 4 + 2 * 2 * (size_t)(Bw + 16) + 64;
+  return fl * 4 + 2 * 2 * (size_t)(Bw + 16) + 192;
 }
 
 // Cholesky of the diagonal tile (K, K) by one warp: lane r < 16 holds row r.  Columns >= n (the
@@ -228,10 +228,10 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   float* dvec = wblk + Bw;
   unsigned short* qlist = reinterpret_cast<unsigned short*>(dvec + Bw);
   unsigned short* klist = qlist + Bw + 16;
-  unsigned* scratch = reinterpret_cast<unsigned*>(klist + Bw + 16);  // 16 words
-  unsigned* warp_sums = scratch;          // [8]
-  unsigned* s_counter = scratch + 9;
-  unsigned* s_bad = scratch + 10;
+  unsigned* scratch = reinterpret_cast<unsigned*>(klist + Bw + 16);  // 48 words
+  unsigned* warp_sums = scratch;          // [32]
+  unsigned* s_counter = scratch + 32;
+  unsigned* s_bad = scratch + 33;
 
   int cnt0, cnt1;
   if (row_lists) {
@@ -315,16 +315,23 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     __syncthreads();
     // ---- gather the lower triangle of M[sel, sel], the right-hand-side row n, identity padding
     {
-      const int r = tid >> 4, k = tid & 15;
+      // 256 threads fill one tile; the CTA's groups of 256 threads take tiles round-robin
+      constexpr int GROUPS = CTA_THREADS / 256;
+      const int r = (tid & 255) >> 4, k = tid & 15, grp = tid >> 8;
       const int ntiles = (T * (T + 1)) >> 1;
       int I = 0, J = 0;
-      for (int t0 = 0; t0 < ntiles; t0 += 8) {  // eight loads in flight per thread
+      for (int g = 0; g < grp; ++g)
+        if (++J > I) {
+          ++I;
+          J = 0;
+        }
+      for (int t0 = grp; t0 < ntiles; t0 += 8 * GROUPS) {  // eight loads in flight per thread
         float v[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int i = 16 * I + r, j = 16 * J + k;
           float x;
-          if (t0 + u >= ntiles)
+          if (t0 + u * GROUPS >= ntiles)
             x = 0.f;
           else if (i < n)
             x = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
@@ -333,14 +340,16 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           else
             x = i == j ? 1.f : 0.f;
           v[u] = x;
-          if (++J > I) {
-            ++I;
-            J = 0;
-          }
+#pragma unroll
+          for (int g = 0; g < GROUPS; ++g)
+            if (++J > I) {
+              ++I;
+              J = 0;
+            }
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-          if (t0 + u < ntiles) A[((t0 + u) << 8) + elem_off(r, k)] = v[u];
+          if (t0 + u * GROUPS < ntiles) A[((t0 + u * GROUPS) << 8) + elem_off(r, k)] = v[u];
       }
     }
     __syncthreads();
