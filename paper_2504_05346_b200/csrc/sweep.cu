@@ -793,7 +793,7 @@ outlier_rows_kernel(const float* __restrict__ h, int c, int n_out, uint8_t* __re
 
 struct SweepWs {
   float* Wc;   // fp32 working copy when the I/O dtype is not fp32
-  __nv_bfloat16* D;    // [3][c, B] change of the current block (delta) as bf16 planes
+  __nv_bfloat16* D;    // [3][c, g B] change of the current block(s) (delta) as bf16 planes
   float* Ubb;  // [blocks, B, B] per-block matrices
   float* Vbb;
   float* G;
@@ -810,6 +810,15 @@ struct SweepWs {
   unsigned* list_counts;  // [2]
 };
 
+// n:m mode: blocks per group whose far update is applied once per group (the update of a block
+// only has to reach the group's own columns before the next block is masked, because the n:m
+// mask reads nothing but its block).  Groups span 512 columns; small layers gain nothing.
+int lazy_group(int64_t b, int B) {
+  if (b < 2048 || B >= 512) return 1;
+  const int g = 512 / B;
+  return g < 1 ? 1 : (g > 8 ? 8 : g);
+}
+
 // room for one key in eight of the layer (the bracket window holds about three in a hundred)
 size_t cand_capacity(int64_t c, int64_t b) {
   size_t n = (size_t)c * (size_t)b / 8;
@@ -823,7 +832,7 @@ bool carve(SweepWs& w, void* workspace, size_t ws_bytes, int64_t c, int64_t b, i
   Arena ar(workspace, ws_bytes);
   const size_t blocks = (size_t)ceil_div(b, B);
   w.Wc = need_wc ? ar.take<float>((size_t)c * b) : nullptr;
-  w.D = ar.take<__nv_bfloat16>(3 * (size_t)c * B);
+  w.D = ar.take<__nv_bfloat16>(3 * (size_t)c * B * lazy_group(b, B));
   w.Ubb = ar.take<float>(blocks * B * B);
   w.Vbb = ar.take<float>(blocks * B * B);
   w.G = ar.take<float>(blocks * B * B);
@@ -868,10 +877,15 @@ thanos_status_t prepare_blocks(const float* U, int b, int B, const SweepWs& w,
 thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* xnorm,
                            thanos_mode_t mode, int n, int m, int B, int j1, int64_t* r_ext,
                            const SweepWs& w, thanos_stats_t* stats, cudaStream_t stream,
-                           const uint8_t* row_skip = nullptr, int n_skip = 0) {
+                           const uint8_t* row_skip = nullptr, int n_skip = 0, int d_col = 0,
+                           int ldd = 0, int upd_end = -1) {
+  // delta goes to columns [d_col, d_col + Bw) of the plane buffer (leading dimension ldd); the
+  // update is applied to columns [j2, upd_end) of W
   const int Bw = (b - j1 < B) ? b - j1 : B;
   const int j2 = j1 + Bw;
   const int bb = j1 / B;
+  if (ldd == 0) ldd = B;
+  if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
     int hg = c < 148 * 8 ? c : 148 * 8;
@@ -902,22 +916,22 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     THANOS_CHECK_LAUNCH();
   }
   THANOS_TRY(launch_block_solve(Wc, mask, w.G + (size_t)bb * B * B, w.S + (size_t)bb * B * B, B,
-                                w.D, (int64_t)c * B, c, b, j1, Bw, B, s_fixed, w.row_lists,
-                                w.list_counts, stats, stream));
-  if (j2 < b) {
-    // W[:, j2:] += delta P2[j1:j2, j2:]
+                                w.D + d_col, (int64_t)c * ldd, c, b, j1, Bw, ldd, s_fixed,
+                                w.row_lists, w.list_counts, stats, stream));
+  if (j2 < upd_end) {
+    // W[:, j2:upd_end] += delta P2[j1:j2, j2:upd_end]
     TcGemmArgs g;
     g.D = Wc + j2;
     g.ldd = b;
-    g.A = w.D;
-    g.lda = B;
-    g.a_plane = (int64_t)c * B;
+    g.A = w.D + d_col;
+    g.lda = ldd;
+    g.a_plane = (int64_t)c * ldd;
     g.B = w.P2 + (int64_t)j1 * b + j2;
     g.ldb = b;
     g.b_plane = (int64_t)b * b;
     g.b_kmajor = 0;
     g.M = c;
-    g.N = b - j2;
+    g.N = upd_end - j2;
     g.K = Bw;
     g.alpha = 1.f;
     g.accumulate = 1;
@@ -933,7 +947,7 @@ size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dty
   size_t t = 0;
   const size_t blocks = (size_t)ceil_div(b, B);
   if (dtype != THANOS_F32) t += round_up((size_t)c * b * sizeof(float), 256);
-  t += round_up(3 * (size_t)c * B * sizeof(__nv_bfloat16), 256);
+  t += round_up(3 * (size_t)c * B * lazy_group(b, B) * sizeof(__nv_bfloat16), 256);
   t += 4 * round_up(blocks * B * B * sizeof(float), 256);
   t += round_up(3 * (size_t)b * b * sizeof(__nv_bfloat16), 256) + 256;
   t += round_up(HIST_BINS * sizeof(unsigned), 256);
@@ -1088,9 +1102,44 @@ thanos_status_t prune_layer_core(const void* W_in, void* W_out, uint8_t* mask_ou
   init_sweep_kernel<<<1, 1, 0, stream>>>(w.st, stats, r);
   THANOS_CHECK_LAUNCH();
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
-  for (int64_t j1 = 0; j1 < b; j1 += B) {
-    THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr, w,
-                          stats, stream, row_skip, n_skip));
+  const int grp = mode == THANOS_NM ? lazy_group(b, B) : 1;
+  if (grp == 1) {
+    for (int64_t j1 = 0; j1 < b; j1 += B) {
+      THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr,
+                            w, stats, stream, row_skip, n_skip));
+    }
+  } else {
+    // n:m: the blocks of a group update the group's columns at once and everything to the right
+    // of the group by one product over the whole group (K = grp B), which reads and writes
+    // those weights once per group instead of once per block
+    const int ldd = grp * B;
+    for (int64_t g0 = 0; g0 < b; g0 += ldd) {
+      const int64_t g_end = g0 + ldd < b ? g0 + ldd : b;
+      for (int64_t j1 = g0; j1 < g_end; j1 += B) {
+        THANOS_TRY(block_step(Wc, mask_out, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, nullptr,
+                              w, stats, stream, row_skip, n_skip, (int)(j1 - g0), ldd,
+                              (int)g_end));
+      }
+      if (g_end < b) {
+        TcGemmArgs g;
+        g.D = Wc + g_end;
+        g.ldd = b;
+        g.A = w.D;
+        g.lda = ldd;
+        g.a_plane = c * ldd;
+        g.B = w.P2 + g0 * b + g_end;
+        g.ldb = b;
+        g.b_plane = b * b;
+        g.b_kmajor = 0;
+        g.M = (int)c;
+        g.N = (int)(b - g_end);
+        g.K = (int)(g_end - g0);
+        g.alpha = 1.f;
+        g.accumulate = 1;
+        g.status = w.tc_status;
+        THANOS_TRY(tc_gemm_split3(g, stream));
+      }
+    }
   }
   fold_tc_status_kernel<<<1, 1, 0, stream>>>(stats, w.tc_status);
   THANOS_CHECK_LAUNCH();

@@ -265,6 +265,8 @@ SWEEP_CASES = [
     ("b512_unstr70", 160, 1024, 4096, "bf16", "student_t4", "unstructured", 0.7, 0, 0, 512, 0.3),
     ("b400_unstr", 90, 1200, 4096, "f32", "normal", "unstructured", 0.45, 0, 0, 400, 0.5),
     ("b512_4of8", 200, 512, 4096, "bf16", "student_t4", "nm", 0.0, 4, 8, 512, 0.0),
+    ("grouped_2of4", 96, 2304, 4096, "f32", "student_t4", "nm", 0.0, 2, 4, 128, 0.3),
+    ("grouped_4of8_b256", 72, 2176, 4096, "bf16", "normal", "nm", 0.0, 4, 8, 256, 0.5),
 ]
 
 
