@@ -667,3 +667,30 @@ def test_structured_full_size_sampled_rows(T):
     Wr = O.structured_update_rows(W64[rows], rm, O.damped(H64, 0.01))
     Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
     assert PU.rel_fro(Wg[rows], Wr) <= PU.TOL_W_BF16
+
+
+def test_structured_edges_and_errors(T):
+    """One row, the smallest width, a single removed column; rejected arguments leave the
+    context usable."""
+    rng = torch.Generator().manual_seed(5)
+    for c, b, p in ((1, 8, 0.5), (3, 16, 1.0 / 16), (5, 24, 0.9)):
+        X = torch.randn((256, b), generator=rng)
+        H = _gpu_hessian(T, X.to(DEV))
+        U, xn = T.prepare_inverse(H, 0.01)
+        W = torch.randn((c, b), generator=rng).to(DEV)
+        Wp, colrm, flags, st = T.prune_layer_structured(W, U, xn, p)
+        Wo, rm_o, _, _ = O.thanos_structured(_np64(W), None, p, 0.0, 0.01, H=_np64(H))
+        assert np.array_equal(colrm.cpu().numpy().astype(bool), rm_o)
+        assert int(flags.sum()) == 0 and st.n_pruned == int(rm_o.sum()) * c
+        assert PU.rel_fro(_np64(Wp), Wo) <= PU.TOL_W_F32
+    with pytest.raises(T.ThanosError) as e:      # ceil(p b / (1 - alpha)) >= b
+        T.prune_layer_structured(W, U, xn, 0.6, alpha=0.5, H=H)
+    assert e.value.code == 1
+    with pytest.raises(ValueError):              # outlier rows need the Hessian
+        T.prune_layer_structured(W, U, xn, 0.25, alpha=0.2)
+    with pytest.raises(T.ThanosError) as e:
+        T.prune_layer_structured(W, U, xn, 0.25,
+                                 workspace=torch.empty(512, dtype=torch.uint8, device=DEV))
+    assert e.value.code == 5
+    Wp, colrm, flags, st = T.prune_layer_structured(W, U, xn, 0.25)
+    assert st.status == 0 and int(colrm.sum()) == 6
