@@ -30,18 +30,19 @@ def block_threshold(W_before, xnorm, j1, mask_block_oracle, r_before):
     return float(np.partition(S.ravel(), r_before - 1)[r_before - 1]), S
 
 
-def classify_unstructured_block(mask_gpu_blk, mask_or_blk, S_blk, tau):
+def classify_unstructured_block(mask_gpu_blk, mask_or_blk, S_blk, tau, tie_rel=None):
     """Split mask differences of one block into near-ties (oracle score within TIE_REL of the
     block threshold, relative) and real mismatches.  Returns (n_near_tie, n_bad)."""
     diff = mask_gpu_blk != mask_or_blk
     if not diff.any():
         return 0, 0
     s = S_blk[diff]
-    near = np.abs(s - tau) <= TIE_REL * max(tau, 1e-300)
+    tie_rel = TIE_REL if tie_rel is None else tie_rel
+    near = np.abs(s - tau) <= tie_rel * max(tau, 1e-300)
     return int(near.sum()), int((~near).sum())
 
 
-def classify_nm_block(mask_gpu_blk, mask_or_blk, S_blk, n, m):
+def classify_nm_block(mask_gpu_blk, mask_or_blk, S_blk, n, m, tie_rel=None):
     """n:m: a difference inside a group is a near-tie if the group's n-th and (n+1)-th smallest
     oracle scores are within TIE_REL (relative)."""
     c, w = S_blk.shape
@@ -57,7 +58,7 @@ def classify_nm_block(mask_gpu_blk, mask_or_blk, S_blk, n, m):
         s = np.sort(S_blk[i, g * m:(g + 1) * m])
         gap = abs(s[n] - s[n - 1])
         cnt = int(diff[i, g * m:(g + 1) * m].sum())
-        if gap <= TIE_REL * max(s[n], 1e-300):
+        if gap <= (TIE_REL if tie_rel is None else tie_rel) * max(s[n], 1e-300):
             near += cnt
         else:
             bad += cnt

@@ -162,7 +162,7 @@ def _oracle_sweep(W64, H64, mode, p, n, m, B, damp, literal):
     return Wo, Mo, steps
 
 
-def _check_sweep(T, W, H, mode, p, n, m, B, damp, tolW, literal=True, tolD=2e-3):
+def _check_sweep(T, W, H, mode, p, n, m, B, damp, tolW, literal=True, tolD=2e-3, tie_rel=None):
     """Runs prepare_inverse + prune_layer on (W, H) and the oracle on the same H; returns
     diagnostics after asserting the parity protocol."""
     c, b = W.shape
@@ -198,10 +198,10 @@ def _check_sweep(T, W, H, mode, p, n, m, B, damp, tolW, literal=True, tolD=2e-3)
                 if mode == "unstructured":
                     tau, S = PU.block_threshold(stp["W_before"], xn64, j1, stp["mask"], r)
                     near, bad = PU.classify_unstructured_block(Mg[:, j1:j2], stp["mask"],
-                                                               S[:, : j2 - j1], tau)
+                                                               S[:, : j2 - j1], tau, tie_rel)
                 else:
                     S = np.abs(stp["W_before"][:, j1:j2]) * xn64[None, j1:j2]
-                    near, bad = PU.classify_nm_block(Mg[:, j1:j2], stp["mask"], S, n, m)
+                    near, bad = PU.classify_nm_block(Mg[:, j1:j2], stp["mask"], S, n, m, tie_rel)
                 break
             r -= int(stp["mask"].sum())
         assert bad == 0, "mask mismatch that is not a near-tie: %d (near-ties %d)" % (bad, near)
@@ -694,3 +694,48 @@ def test_structured_edges_and_errors(T):
     assert e.value.code == 5
     Wp, colrm, flags, st = T.prune_layer_structured(W, U, xn, 0.25)
     assert st.status == 0 and int(colrm.sum()) == 6
+
+
+# ------------------------------------------------------------------------------ config shapes
+@pytest.mark.parametrize("layer", [0, 4, 5], ids=["q_768x768", "fc1_3072x768", "fc2_768x3072"])
+def test_opt125m_layer_shapes_full_oracle(T, layer):
+    """The OPT-125M-shaped layers (2:4, B = 128, fp32) against the oracle's whole sweep, with the
+    Hessian from 8192 of the configuration's tokens.  In the 3072-wide layer a group is decided
+    up to 23 block updates after the start: the fp32 working copy has then drifted about 1e-5
+    (relative) from the float64 one, so a flip between two scores closer than 1e-4 counts as a
+    near-tie there (seen: one group with a gap of 1.2e-5 in block 22)."""
+    cfg = WL.CONFIGS["opt125m"]
+    L = cfg.layers[layer]
+    W = WL.config_weight(cfg, layer)
+    Xt = WL.config_activations(cfg, L.input_id, L.b, a=8192)
+    H = _gpu_hessian(T, Xt, chunks=2)
+    out = _check_sweep(T, W, H, "nm", 0.0, cfg.n, cfg.m, cfg.B, cfg.damp_rel, PU.TOL_W_F32,
+                       tie_rel=1e-4 if L.b > 1024 else None)
+    assert out["mismatch"] <= 4
+
+
+@pytest.mark.parametrize("mode", ["nm", "unstructured"])
+def test_llama2_70b_width_8192_sampled_rows(T, mode):
+    """The 8192-wide projection of the LLaMA-2-70B-shaped set (2:4 and 60 % unstructured,
+    B = 128, bf16) with 512 rows: counts, exact zeros, and a float64 replay of sampled rows under
+    the GPU's mask."""
+    cfg = WL.CONFIGS["llama2_70b"]
+    c, b, B = 512, 8192, cfg.B
+    W = WL.make_weight(c, b, "bf16", seed=cfg.seed, layer_index=0, device=DEV)
+    Xd = WL.config_activations(cfg, 0, b, device=DEV, a=12288)
+    H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(H, Xd)
+    U, xn = T.prepare_inverse(H, cfg.damp_rel)
+    if mode == "nm":
+        Wp, M, st = T.prune_layer(W, U, xn, T.NM, n=2, m=4, B=B)
+        assert bool((M.view(c, b // 4, 4).sum(dim=2) == 2).all())
+    else:
+        Wp, M, st = T.prune_layer(W, U, xn, T.UNSTRUCTURED, p=0.6, B=B)
+        assert st.n_pruned == PU.expected_removed(0.6, c, b) and st.r_left == 0
+        assert st.select_misses <= 2
+    assert st.n_blocks == b // B and bool((Wp[M.bool()] == 0).all())
+    Hd = O.damped(_np64(H), cfg.damp_rel)
+    rows = np.array([0, 255, 511])
+    Wr = O.replay_rows(_np64(W)[rows], M.cpu().numpy()[rows], Hd, B)
+    Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
+    assert PU.rel_fro(_np64(Wp)[rows], Wr) <= PU.TOL_W_BF16
