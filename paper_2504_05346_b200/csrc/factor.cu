@@ -11,13 +11,13 @@
 // whose levels are tensor-core products as well.
 #include "simt_gemm.cuh"
 #include "tc_gemm.cuh"
+#include "tile_ops.cuh"
 
 namespace thanos {
 
 namespace {
 
 constexpr int NB = 128;
-constexpr int DLD = NB + 4;  // row stride of the diagonal-block scratch (odd multiple of 16 bytes)
 
 // ---- mean(diag H) -> lambda, xnorm ---------------------------------------------------------
 __global__ void __launch_bounds__(1024)
@@ -58,116 +58,121 @@ __global__ void copy_damped_upper_kernel(const float* __restrict__ H, float* __r
 //      U22 = inv(V22).  One CTA.  With the rows and columns reversed this is an ordinary lower
 //      Cholesky L; n identity rows appended below the block turn into L^{-T} under the same
 //      elimination, which gives the inverse without a second pass.
-//      Left-looking in panels of 8 columns.  Two threads share a row and split the contraction
-//      range in alternating runs of 16 columns; every thread factors the 8 x 8 diagonal piece
-//      itself (reciprocal square roots by one Newton step on the hardware estimate).
-constexpr int DIAG_THREADS = 4 * NB;
+//      The stacked matrix [reversed block; identity] lives in shared memory as 16 x 16 tiles
+//      (2 Tn tile rows, Tn tile columns).  Right-looking: per tile column K the rows of the panel
+//      are solved one thread per row, the trailing tiles are updated one warp per tile from a
+//      shared counter, and warp 0 first brings the next diagonal tile up to date and factors it
+//      (reciprocal square roots by one Newton step on the hardware estimate).  Identity row j
+//      is zero left of column j, so its tiles join in from tile column j / 16 on.
+constexpr int DIAG_THREADS = 512;
+constexpr int DIAG_TILES = NB / 16;
+constexpr int DIAG_SMEM = (2 * DIAG_TILES * DIAG_TILES * 256 + NB + 16) * (int)sizeof(float);
 
-__global__ void __launch_bounds__(DIAG_THREADS)
+__global__ void __launch_bounds__(DIAG_THREADS, 1)
 diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* __restrict__ Up,
                   int64_t plane, int b, int k0, int n, int32_t* __restrict__ status) {
   extern __shared__ __align__(16) float dsm[];
-  float* L = dsm;                       // [2 n][DLD]
-  float* dblk = dsm + 2 * NB * DLD;     // [8][8]
+  const int Tn = (n + 15) >> 4;
+  float* A = dsm;                                   // tile (I, J) at (I Tn + J) * 256
+  float* invd = dsm + 2 * DIAG_TILES * DIAG_TILES * 256;  // [NB]
+  unsigned* s_counter = reinterpret_cast<unsigned*>(invd + NB);
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
-  // reversed lower triangle of the block, then the identity
-  for (int i = warp; i < n; i += DIAG_THREADS / 32) {
-    const float* src = V + (int64_t)(k0 + n - 1 - i) * b + k0;
-    for (int c4 = lane * 4; c4 < n; c4 += 128) {
-      const float4 v = *reinterpret_cast<const float4*>(src + c4);
-      const float e[4] = {v.x, v.y, v.z, v.w};
+  auto tile_at = [&](int I, int J) { return A + ((I * Tn + J) << 8); };
+  // zeros, with ones on the diagonal of the padding and of the identity rows ...
+  for (int q = tid; q < 2 * Tn * Tn * 64; q += DIAG_THREADS) {
+    const int t = q >> 6, r = (q >> 2) & 15, c = q & 3;
+    const int I = t / Tn, J = t - I * Tn;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int d = r - 4 * c;  // the chunk holds the tile's diagonal element of row r at position d
+    const bool diag_tile = I >= Tn ? (I - Tn == J) : (I == J && 16 * I + r >= n);
+    if (diag_tile && d >= 0 && d < 4) {
+      if (d == 0) v.x = 1.f;
+      if (d == 1) v.y = 1.f;
+      if (d == 2) v.z = 1.f;
+      if (d == 3) v.w = 1.f;
+    }
+    *reinterpret_cast<float4*>(A + (t << 8) + tile::chunk_off(r, c)) = v;
+  }
+  __syncthreads();
+  // ... then the reversed lower triangle of the block: a warp takes rows i, i + 16, ..., all of
+  // its loads first
+  {
+    float4 v[NB / (DIAG_THREADS / 32)];
+    const int c4 = lane * 4;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = n - 1 - (c4 + u);
-        L[i * DLD + j] = (j <= i) ? e[u] : 0.f;
-        L[(n + i) * DLD + j] = (i == j) ? 1.f : 0.f;
+    for (int u = 0; u < NB / (DIAG_THREADS / 32); ++u) {
+      const int i = warp + u * (DIAG_THREADS / 32);
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < n && c4 < n)
+        v[u] = *reinterpret_cast<const float4*>(V + (int64_t)(k0 + n - 1 - i) * b + k0 + c4);
+    }
+#pragma unroll
+    for (int u = 0; u < NB / (DIAG_THREADS / 32); ++u) {
+      const int i = warp + u * (DIAG_THREADS / 32);
+      if (i < n && c4 < n) {
+        const float e4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const int j = n - 1 - (c4 + w);
+          if (j <= i) tile_at(i >> 4, j >> 4)[tile::elem_off(i & 15, j & 15)] = e4[w];
+        }
       }
     }
   }
   __syncthreads();
-  const int r = tid >> 1;
-  const int half = tid & 1;
-  const bool is_row = r < 2 * n;
-  float* Lr = L + (is_row ? r : 0) * DLD;
-  // identity row j is zero left of column j: its products start there (rounded down to 32)
-  const int first_nz = (r >= n) ? ((r - n) & ~31) : 0;
-  for (int c0 = 0; c0 < n; c0 += 8) {
-    const bool active = is_row && r >= c0;
-    float acc[8];
-    if (half == 0) {
-      const float4 lo = *reinterpret_cast<const float4*>(Lr + c0);
-      const float4 hi = *reinterpret_cast<const float4*>(Lr + c0 + 4);
-      acc[0] = lo.x; acc[1] = lo.y; acc[2] = lo.z; acc[3] = lo.w;
-      acc[4] = hi.x; acc[5] = hi.y; acc[6] = hi.z; acc[7] = hi.w;
-    } else {
-#pragma unroll
-      for (int w = 0; w < 8; ++w) acc[w] = 0.f;
-    }
-    if (active) {
-      const float* Pb = L + c0 * DLD;
-      for (int kk = first_nz + 16 * half; kk < c0; kk += 32) {
-        const int kend = kk + 16 < c0 ? kk + 16 : c0;
-        for (int k = kk; k < kend; k += 4) {
-          const float4 av = *reinterpret_cast<const float4*>(Lr + k);
-#pragma unroll
-          for (int w = 0; w < 8; ++w) {
-            const float4 bv = *reinterpret_cast<const float4*>(Pb + w * DLD + k);
-            acc[w] = fmaf(-av.x, bv.x, acc[w]);
-            acc[w] = fmaf(-av.y, bv.y, acc[w]);
-            acc[w] = fmaf(-av.z, bv.z, acc[w]);
-            acc[w] = fmaf(-av.w, bv.w, acc[w]);
-          }
-        }
+  int bad = -1;
+  if (warp == 0) bad = tile::factor_diag_tile<true>(tile_at(0, 0), invd, 0, n, lane);
+  __syncthreads();
+  for (int K = 0; K < Tn; ++K) {
+    const int m = Tn - K - 1;  // tile rows of the block below the diagonal tile
+    if (tid == 0) *s_counter = 1;
+    // panel: the block's rows below the diagonal tile and the identity rows 0 .. 16 K + 15
+    {
+      const float* Lk = tile_at(K, K);
+      for (int ii = tid; ii < 16 * (m + K + 1); ii += DIAG_THREADS) {
+        const int tr = ii >> 4, r = ii & 15;
+        const int I = tr < m ? K + 1 + tr : Tn + (tr - m);
+        tile::panel_row_solve(tile_at(I, K), r, Lk, invd + 16 * K);
       }
-    }
-#pragma unroll
-    for (int w = 0; w < 8; ++w) acc[w] += __shfl_xor_sync(0xffffffffu, acc[w], 1);
-    if (half == 0 && r >= c0 && r < c0 + 8) {
-#pragma unroll
-      for (int w = 0; w < 8; ++w) dblk[(r - c0) * 8 + w] = acc[w];
     }
     __syncthreads();
-    // 8 x 8 Cholesky of the diagonal piece, in registers, by every thread
-    float ld[8][8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-#pragma unroll
-      for (int j = 0; j <= i; ++j) ld[i][j] = dblk[i * 8 + j];
-    float rinv[8];
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      float d = ld[w][w];
-      if (!(d > 0.f) || !isfinite(d)) {
-        if (tid == 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + n - 1 - (c0 + w));
-        d = 1.f;
+    if (warp == 0 && K + 1 < Tn) {
+      float* Ct = tile_at(K + 1, K + 1);
+      tile::tile_update(Ct, tile_at(K + 1, K), tile_at(K + 1, K), lane);
+      __syncwarp();
+      const int bd = tile::factor_diag_tile<true>(Ct, invd, 16 * (K + 1), n, lane);
+      if (bad < 0) bad = bd;
+    }
+    {
+      // targets: the m (m + 1) / 2 tiles (I, J), K < J <= I, of the block (index 0 is the next
+      // diagonal tile, done above), then the (K + 1) m tiles of the identity rows
+      const int ntop = (m * (m + 1)) >> 1;
+      const int total = ntop + (K + 1) * m;
+      for (;;) {
+        unsigned u = 0;
+        if (lane == 0) u = atomicAdd(s_counter, 1u);
+        u = __shfl_sync(0xffffffffu, u, 0);
+        if ((int)u >= total) break;
+        int I, J;
+        if ((int)u < ntop) {
+          int Ip = (int)((sqrtf(8.f * (float)u + 1.f) - 1.f) * 0.5f);
+          while (((Ip + 1) * (Ip + 2) >> 1) <= (int)u) ++Ip;
+          while (((Ip * (Ip + 1)) >> 1) > (int)u) --Ip;
+          I = K + 1 + Ip;
+          J = K + 1 + (int)u - ((Ip * (Ip + 1)) >> 1);
+        } else {
+          const int v = (int)u - ntop;
+          I = Tn + v / m;
+          J = K + 1 + v % m;
+        }
+        tile::tile_update(tile_at(I, J), tile_at(I, K), tile_at(J, K), lane);
       }
-      float ri = rsqrtf(d);
-      ri = ri * fmaf(-0.5f * d, ri * ri, 1.5f);
-      rinv[w] = ri;
-#pragma unroll
-      for (int v = w; v < 8; ++v) ld[v][w] *= ri;
-#pragma unroll
-      for (int v = w + 1; v < 8; ++v)
-#pragma unroll
-        for (int u = w + 1; u <= v; ++u) ld[v][u] = fmaf(-ld[v][w], ld[u][w], ld[v][u]);
-    }
-    // this thread's row: x L_d^T = acc
-    float x[8];
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      float t = acc[w];
-#pragma unroll
-      for (int v = 0; v < w; ++v) t = fmaf(-x[v], ld[w][v], t);
-      x[w] = t * rinv[w];
-    }
-    if (active && half == 0) {
-      *reinterpret_cast<float4*>(Lr + c0) = make_float4(x[0], x[1], x[2], x[3]);
-      *reinterpret_cast<float4*>(Lr + c0 + 4) = make_float4(x[4], x[5], x[6], x[7]);
     }
     __syncthreads();
   }
-  // V22[i][j] = L[n-1-i][n-1-j];  U22[i][j] = inv(L)[n-1-i][n-1-j] = extra row (n-1-j), column n-1-i
+  if (warp == 0 && lane == 0 && bad >= 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + n - 1 - bad);
+  // V22[i][j] = L[n-1-i][n-1-j];  U22[i][j] = inv(L)[n-1-i][n-1-j] = identity row (n-1-j), column n-1-i
   for (int i = warp; i < n; i += DIAG_THREADS / 32) {
     for (int c4 = lane * 4; c4 < n; c4 += 128) {
       float u4[4];
@@ -177,8 +182,9 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
         const int j = c4 + e;
         float u = 0.f;
         if (j >= i) {
-          V[o + e] = L[(n - 1 - i) * DLD + (n - 1 - j)];
-          u = L[(n + n - 1 - j) * DLD + (n - 1 - i)];
+          const int li = n - 1 - i, lj = n - 1 - j;  // lj <= li
+          V[o + e] = tile_at(li >> 4, lj >> 4)[tile::elem_off(li & 15, lj & 15)];
+          u = tile_at(Tn + (lj >> 4), li >> 4)[tile::elem_off(lj & 15, li & 15)];
         }
         u4[e] = u;
       }
@@ -255,7 +261,6 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
   THANOS_CUDA(cudaMemsetAsync(w.Up, 0, 3 * (size_t)plane * sizeof(__nv_bfloat16), stream));
   THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
 
-  constexpr int DIAG_SMEM = (2 * NB * DLD + 64) * (int)sizeof(float);
   {
     static std::atomic<unsigned long long> done{0};
     THANOS_CUDA(ensure_max_dyn_smem(diag_block_kernel, DIAG_SMEM, done));

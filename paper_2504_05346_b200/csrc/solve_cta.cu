@@ -11,10 +11,15 @@
 // next diagonal tile first, which takes the only serial step off the critical path.  Blocked
 // back substitution L^T x = y, then the change of the block's weights as in the small kernel.
 #include "common.cuh"
+#include "tile_ops.cuh"
 
 namespace thanos {
 
 namespace {
+
+using tile::chunk_off;
+using tile::elem_off;
+using tile::tile_update;
 
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int CTA_THREADS = 512;
@@ -32,92 +37,10 @@ __device__ __forceinline__ void put_split3(__nv_bfloat16* __restrict__ p, int64_
 
 // tile (I, J), J <= I, of the lower triangle; 256 floats each
 __device__ __forceinline__ int tile_base(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
-// 16-byte chunk c of row r sits at chunk position c ^ ((r >> 1) & 3)
-__device__ __forceinline__ int chunk_off(int r, int c) { return (r << 4) + (((c ^ (r >> 1)) & 3) << 2); }
-__device__ __forceinline__ int elem_off(int r, int k) { return chunk_off(r, k >> 2) + (k & 3); }
-
 __host__ __device__ inline size_t cta_smem_bytes(int tiles, int Bw) {
   // tiles, invd / xs / rhs [16 tiles + 16 each], wblk / dvec [Bw], two index lists, scan scratch
   const size_t fl = (size_t)(tiles * (tiles + 1) / 2) * 256 + 3 * (16 * (size_t)tiles + 16) + 2 * (size_t)Bw;
   return fl * 4 + 2 * 2 * (size_t)(Bw + 16) + 192;
-}
-
-// Cholesky of the diagonal tile (K, K) by one warp: lane r < 16 holds row r.  Columns >= n (the
-// right-hand-side row and the identity padding) get pivot 1.
-__device__ __forceinline__ bool factor_diag_tile(float* __restrict__ Tt, float* __restrict__ invd,
-                                                 int col0, int n, int lane) {
-  const int r = lane & 15;
-  float a[16];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const float4 v = *reinterpret_cast<const float4*>(Tt + chunk_off(r, c));
-    a[4 * c] = v.x; a[4 * c + 1] = v.y; a[4 * c + 2] = v.z; a[4 * c + 3] = v.w;
-  }
-  bool bad = false;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    float dj = __shfl_sync(FULL, a[j], j);
-    if (col0 + j < n) {
-      if (!(dj > 0.f) || !isfinite(dj)) {
-        bad = true;
-        dj = 1.f;
-      }
-    } else {
-      dj = 1.f;
-    }
-    const float rinv = rsqrtf(dj);
-    if (lane == 0) invd[col0 + j] = rinv;
-    a[j] *= rinv;
-#pragma unroll
-    for (int v = j + 1; v < 16; ++v) {
-      const float lvj = __shfl_sync(FULL, a[j], v);
-      a[v] = fmaf(-a[j], lvj, a[v]);
-    }
-  }
-  if (lane < 16) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-      *reinterpret_cast<float4*>(Tt + chunk_off(r, c)) =
-          make_float4(a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
-  }
-  __syncwarp();
-  return bad;
-}
-
-// C -= A B^T for 16 x 16 tiles by one warp: lane (lr, lc) owns rows lr, lr + 8 and columns
-// lc, lc + 4, lc + 8, lc + 12.
-__device__ __forceinline__ void tile_update(float* __restrict__ Ct, const float* __restrict__ At,
-                                            const float* __restrict__ Bt, int lane) {
-  const int lr = lane >> 2, lc = lane & 3;
-  float acc[2][4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) acc[0][i] = acc[1][i] = 0.f;
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const float4 a0 = *reinterpret_cast<const float4*>(At + chunk_off(lr, c));
-    const float4 a1 = *reinterpret_cast<const float4*>(At + chunk_off(lr + 8, c));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float4 bv = *reinterpret_cast<const float4*>(Bt + chunk_off(lc + 4 * i, c));
-      acc[0][i] = fmaf(a0.x, bv.x, acc[0][i]);
-      acc[0][i] = fmaf(a0.y, bv.y, acc[0][i]);
-      acc[0][i] = fmaf(a0.z, bv.z, acc[0][i]);
-      acc[0][i] = fmaf(a0.w, bv.w, acc[0][i]);
-      acc[1][i] = fmaf(a1.x, bv.x, acc[1][i]);
-      acc[1][i] = fmaf(a1.y, bv.y, acc[1][i]);
-      acc[1][i] = fmaf(a1.z, bv.z, acc[1][i]);
-      acc[1][i] = fmaf(a1.w, bv.w, acc[1][i]);
-    }
-  }
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int r = lr + 8 * h;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float* p = Ct + chunk_off(r, i) + lc;  // column lc + 4 i: chunk i, element lc
-      *p -= acc[h][i];
-    }
-  }
 }
 
 // 2 x 2 target tiles (I0 + di, J0 + dj) of step K at once: C_IJ -= L_IK L_JK^T.  Lane (lr, lc)
@@ -354,7 +277,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     }
     __syncthreads();
     bool bad = false;
-    if (warp == 0) bad = factor_diag_tile(A + tile_base(0, 0), invd, 0, n, lane);
+    if (warp == 0) bad = tile::factor_diag_tile<false>(A + tile_base(0, 0), invd, 0, n, lane) >= 0;
     __syncthreads();
     // ---- right-looking tile Cholesky
     for (int K = 0; K < Tf; ++K) {
@@ -365,30 +288,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         const float* Lk = A + tile_base(K, K);
         for (int ii = tid; ii < 16 * m; ii += CTA_THREADS) {
           const int I = K + 1 + (ii >> 4), r = ii & 15;
-          float* arow = A + tile_base(I, K);
-          float x[16];
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            const float4 v = *reinterpret_cast<const float4*>(arow + chunk_off(r, cc));
-            x[4 * cc] = v.x; x[4 * cc + 1] = v.y; x[4 * cc + 2] = v.z; x[4 * cc + 3] = v.w;
-          }
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float l[16];
-#pragma unroll
-            for (int cc = 0; cc <= ((j - 1) >> 2) && j > 0; ++cc) {
-              const float4 v = *reinterpret_cast<const float4*>(Lk + chunk_off(j, cc));
-              l[4 * cc] = v.x; l[4 * cc + 1] = v.y; l[4 * cc + 2] = v.z; l[4 * cc + 3] = v.w;
-            }
-            float acc = x[j];
-#pragma unroll
-            for (int mm = 0; mm < j; ++mm) acc = fmaf(-x[mm], l[mm], acc);
-            x[j] = acc * invd[16 * K + j];
-          }
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc)
-            *reinterpret_cast<float4*>(arow + chunk_off(r, cc)) =
-                make_float4(x[4 * cc], x[4 * cc + 1], x[4 * cc + 2], x[4 * cc + 3]);
+          tile::panel_row_solve(A + tile_base(I, K), r, Lk, invd + 16 * K);
         }
       }
       __syncthreads();
@@ -398,7 +298,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         const float* At = A + tile_base(K + 1, K);
         tile_update(Ct, At, At, lane);
         __syncwarp();
-        bad |= factor_diag_tile(Ct, invd, 16 * (K + 1), n, lane);
+        bad |= tile::factor_diag_tile<false>(Ct, invd, 16 * (K + 1), n, lane) >= 0;
       }
       {
         // the m x m lower triangle of targets in 2 x 2 groups (I', J') in row-major order,
