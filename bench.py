@@ -359,21 +359,51 @@ def run_e2e(T, cfg, a, dev, dt, margs, world, args):
     host_m = [torch.empty(w.shape, dtype=torch.uint8).pin_memory() for w in host_w]
     torch.cuda.empty_cache()
     arena_bytes = max(T.workspace_bytes(3, L.c, L.b, cfg.B, dt) for L in cfg.layers)
-    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
     h2d = sum(x.numel() * x.element_size() for x in host_in.values()) + \
         sum(w.numel() * w.element_size() for w in host_w)
     d2h = sum(w.numel() * w.element_size() + w.numel() + 64 for w in host_w)
 
+    # Layers that share an input share its factor, so they stay together and in order; the
+    # groups are dealt to host threads (largest first, to the lighter thread), each with its own
+    # stream and arena, so that one group's copies overlap another group's kernels.
+    groups = {}
+    for i, L in enumerate(cfg.layers):
+        groups.setdefault(L.input_id, []).append(i)
+    n_workers = max(1, min(args.e2e_workers, len(groups)))
+    load = [0] * n_workers
+    plan = [[] for _ in range(n_workers)]
+    for gid in sorted(groups, key=lambda g: -host_in[g].numel()):
+        k = load.index(min(load))
+        plan[k].append(gid)
+        load[k] += host_in[gid].numel() + sum(host_w[i].numel() for i in groups[gid])
+    arenas = [torch.empty(arena_bytes, dtype=torch.uint8, device=dev) for _ in range(n_workers)]
+    streams = [torch.cuda.Stream(device=dev) for _ in range(n_workers)]
+    errors = []
+
+    def work(k):
+        try:
+            torch.cuda.set_device(dev)
+            for gid in plan[k]:
+                for pos, i in enumerate(groups[gid]):
+                    reuse = pos > 0
+                    T.prune_layer_host(host_w[i], None if reuse else host_in[gid], cfg.damp_rel,
+                                       B=cfg.B, arena=arenas[k], reuse_factor=reuse,
+                                       out=host_o[i], mask=host_m[i], stream=streams[k], **margs)
+        except Exception as e:  # reported by the caller's thread
+            errors.append(e)
+
     def step():
-        seen = None
-        order = sorted(range(len(cfg.layers)), key=lambda i: cfg.layers[i].input_id)
-        for i in order:
-            L = cfg.layers[i]
-            reuse = seen == L.input_id
-            T.prune_layer_host(host_w[i], None if reuse else host_in[L.input_id], cfg.damp_rel,
-                               B=cfg.B, arena=arena, reuse_factor=reuse, out=host_o[i],
-                               mask=host_m[i], **margs)
-            seen = L.input_id
+        import threading
+        if n_workers == 1:
+            work(0)
+        else:
+            ts = [threading.Thread(target=work, args=(k,)) for k in range(n_workers)]
+            for t in ts:
+                t.start()
+            for t in ts:
+                t.join()
+        if errors:
+            raise errors[0]
 
     step()  # warm-up
     torch.cuda.synchronize()
@@ -387,7 +417,7 @@ def run_e2e(T, cfg, a, dev, dt, margs, world, args):
     dt_s = max_over_ranks(dt_s, dev)
     return {"value": world * layer_set_weights(cfg) * steps / dt_s, "unit": UNIT,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
-            "ms_per_step": dt_s * 1e3 / steps}
+            "ms_per_step": dt_s * 1e3 / steps, "host_threads": n_workers}
 
 
 # ------------------------------------------------------------------------------------------
@@ -536,6 +566,8 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="issue every call on one stream instead of one stream per input / layer")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-workers", type=int, default=3,
+                    help="host threads (each with a stream and an arena) of the end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
     ap.add_argument("--single-layer", default="", metavar="C,B,A",
