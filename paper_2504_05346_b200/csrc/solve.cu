@@ -17,6 +17,7 @@
 // right-hand side is appended as one more row, so the factorisation L L^T also yields
 // L^{-1} rhs.  Left-looking Cholesky in panels of 8 columns: a lane owns up to NR rows of the
 // panel (8 accumulators each), the 8 x 8 diagonal block is factored with warp shuffles.
+// Systems of 160 unknowns and more go to the CTA-per-row kernel of solve_cta.cu.
 #include "common.cuh"
 
 namespace thanos {
