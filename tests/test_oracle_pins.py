@@ -398,6 +398,8 @@ def test_column_losses_match_the_frobenius_definition():
         assert abs(v[j] - np.linalg.norm(outer, "fro") ** 2) <= 1e-10 * v[j]
     assert O.structured_column_count(0.3, 10, 0.0) == 3
     assert O.structured_column_count(0.3, 10, 0.25) == 4     # ceil(3 / 0.75)
+    assert O.structured_column_count(0.25, 10, 0.0) == 3     # ceil(2.5): rounded up
+    assert O.structured_column_count(0.5, 7, 0.1) == 4       # ceil(3.5 / 0.9) = ceil(3.89)
 
 
 def test_structured_is_the_constrained_least_squares_refit():
