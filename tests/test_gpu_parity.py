@@ -490,10 +490,12 @@ def test_outlier_rows_parity(T, c, b, dtype, n, m, B, alpha):
 
 
 # ------------------------------------------------------------------------------ bench-size
-def test_full_size_layer_sampled_rows(T):
-    """4096 x 4096 bf16 layer, B = 128 (benchmark shape), 50 % unstructured and 2:4: structural
-    invariants on the whole output and a float64 replay of sampled rows under the GPU's mask."""
-    c = b = 4096
+@pytest.mark.parametrize("c", [4096, 11008], ids=["q_4096x4096", "gate_11008x4096"])
+def test_full_size_layer_sampled_rows(T, c):
+    """4096-wide bf16 layers of the benchmark (4096 and 11008 rows), B = 128, 50 % unstructured
+    and 2:4: structural invariants on the whole output and a float64 replay of sampled rows under
+    the GPU's mask."""
+    b = 4096
     B = 128
     W = WL.make_weight(c, b, "bf16", seed=2, layer_index=0, device=DEV)
     Xd = WL.make_activations(16384, b, "bf16", "student_t4", 0.005, 0, 50.0, 2, 0, device=DEV)
@@ -503,7 +505,7 @@ def test_full_size_layer_sampled_rows(T):
     H64 = _np64(H)
     Hd = O.damped(H64, 0.01)
     xn64 = O.feature_norms(H64)
-    rows = np.array([0, 1, 777, 2048, 4095])
+    rows = np.array([0, 1, 777, 2048, c - 1])
     W64 = _np64(W)
     for mode in ("unstructured", "nm"):
         if mode == "unstructured":
