@@ -76,6 +76,17 @@ struct Arena {
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
+// x -> three bf16 planes h = bf16(x), m = bf16(x - h), l = bf16(x - h - m), `plane` elements apart
+// (the operand format of the tensor-core products, see tc_gemm.cuh)
+__device__ __forceinline__ void store_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
+#pragma unroll
+  for (int pl = 0; pl < 3; ++pl) {
+    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
+    p[(int64_t)pl * plane] = hb;
+    d -= __bfloat162float(hb);
+  }
+}
+
 // First device-detected error wins.
 __device__ __forceinline__ void report_error(int32_t* status2, int32_t code, int32_t index) {
   if (atomicCAS(status2, 0, code) == 0) status2[1] = index;

@@ -26,16 +26,6 @@ namespace {
 
 constexpr unsigned FULL = 0xffffffffu;
 
-// delta -> three bf16 planes (h, m, l) for the tensor-core update
-__device__ __forceinline__ void store_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
-#pragma unroll
-  for (int pl = 0; pl < 3; ++pl) {
-    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
-    p[(int64_t)pl * plane] = hb;
-    d -= __bfloat162float(hb);
-  }
-}
-
 __host__ __device__ __forceinline__ int tri_row_off(int r) {
   // rows 8m .. 8m+7 have 8m + 12 floats each (8m + 8 columns plus a 4-float skew)
   const int m = r >> 3, t = r & 7;

@@ -26,15 +26,6 @@ constexpr int CTA_THREADS = 512;
 constexpr int CTA_WARPS = CTA_THREADS / 32;
 constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 - 1 = 319 unknowns
 
-__device__ __forceinline__ void put_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
-#pragma unroll
-  for (int pl = 0; pl < 3; ++pl) {
-    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
-    p[(int64_t)pl * plane] = hb;
-    d -= __bfloat162float(hb);
-  }
-}
-
 // tile (I, J), J <= I, of the lower triangle; 256 floats each
 __device__ __forceinline__ int tile_base(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
 __host__ __device__ inline size_t cta_smem_bytes(int tiles, int Bw) {
@@ -191,7 +182,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     }
     if (tid == 0) *s_bad = 0;
     if (s == 0) {  // nothing removed: the row is not touched in this block (CTA-uniform)
-      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
     if (report_max_s && row == 0 && tid == 0) atomicMax(&stats->max_s, s);
@@ -208,7 +199,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     if ((s > t) != kpath || T > tiles) {
       // cannot happen for lists and launch sizes made by this library
       if (tid == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
-      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
     __syncthreads();
@@ -339,7 +330,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     __syncthreads();
     if (*s_bad) {
       if (tid == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
-      for (int jj = tid; jj < Bw; jj += CTA_THREADS) put_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+      for (int jj = tid; jj < Bw; jj += CTA_THREADS) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
     for (int Kb = Tf - 1; Kb >= 0; --Kb) {
@@ -395,7 +386,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       const float d = dvec[jj];
       const bool removed = mrow[jj] != 0;
       wrow[jj] = removed ? 0.f : wblk[jj] + d;
-      put_split3(D + (int64_t)row * ldd + jj, dplane, d);
+      store_split3(D + (int64_t)row * ldd + jj, dplane, d);
     }
   }
 }

@@ -22,6 +22,8 @@ thanos_status_t outlier_row_flags(const float* Wc, const float* H, int64_t c, in
                                   void* scratch, size_t scratch_bytes, uint8_t** flags_dev,
                                   int32_t* tc_status, cudaStream_t stream);
 size_t prepare_workspace_bytes(int64_t b);
+thanos_status_t convert_to_f32(const __nv_bfloat16* in, float* out, int64_t n, cudaStream_t stream);
+thanos_status_t convert_to_bf16(const float* in, __nv_bfloat16* out, int64_t n, cudaStream_t stream);
 thanos_status_t prepare_inverse_impl(const float* H, int64_t b, float damp_rel, float* factor,
                                      float* xnorm, void* workspace, size_t ws_bytes,
                                      int32_t* status_dev, cudaStream_t stream);
@@ -29,29 +31,6 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b, float damp_rel, 
 namespace {
 
 constexpr int ROW_CHUNK = 64;  // rows per partial sum of the column losses
-
-__device__ __forceinline__ void put_split3(__nv_bfloat16* __restrict__ p, int64_t plane, float d) {
-#pragma unroll
-  for (int pl = 0; pl < 3; ++pl) {
-    const __nv_bfloat16 hb = __float2bfloat16_rn(d);
-    p[(int64_t)pl * plane] = hb;
-    d -= __bfloat162float(hb);
-  }
-}
-
-__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out,
-                                   int64_t n) {
-  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (; i < n; i += stride) out[i] = __bfloat162float(in[i]);
-}
-
-__global__ void f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out,
-                                   int64_t n) {
-  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
-}
 
 // partial[chunk][j] = sum over the pruned rows of the chunk of W_ij^2 (fixed order: the column
 // ranking must not depend on the launch)
@@ -197,7 +176,7 @@ gather_uq_kernel(const float* __restrict__ U, int b, const int* __restrict__ qli
   if (k >= b) return;
   for (int i = ty; i < 32; i += 8) {
     const int aa = a0 + i;
-    if (aa < s_pad) put_split3(planes + (int64_t)aa * b + k, (int64_t)s_pad * b, tile[tx][i]);
+    if (aa < s_pad) store_split3(planes + (int64_t)aa * b + k, (int64_t)s_pad * b, tile[tx][i]);
   }
 }
 
@@ -231,7 +210,7 @@ transpose_split_kernel(const float* __restrict__ in, int n, __nv_bfloat16* __res
   for (int i = ty; i < 32; i += 8) {
     const int orow = c0 + i, ocol = r0 + tx;  // out[orow][ocol] = in[ocol][orow]
     if (orow < n && ocol < n)
-      put_split3(planes + (int64_t)orow * n + ocol, (int64_t)n * n, tile[tx][i]);
+      store_split3(planes + (int64_t)orow * n + ocol, (int64_t)n * n, tile[tx][i]);
   }
 }
 
@@ -244,7 +223,7 @@ gather_wq_kernel(const float* __restrict__ Wc, const uint8_t* __restrict__ flags
   if (a >= s_pad) return;
   const int q = qlist[a];
   const float val = (q >= 0 && !flags[i]) ? Wc[(int64_t)i * b + q] : 0.f;
-  put_split3(planes + (int64_t)i * s_pad + a, (int64_t)c * s_pad, val);
+  store_split3(planes + (int64_t)i * s_pad + a, (int64_t)c * s_pad, val);
 }
 
 // exact zeros in the removed columns of the pruned rows
@@ -374,9 +353,7 @@ thanos_status_t prune_layer_structured_impl(const void* W_in, void* W_out, uint8
   float* Wc;
   if (need_wc) {
     Wc = w.Wc;
-    bf16_to_f32_kernel<<<148 * 8, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(W_in), Wc,
-                                                    nel);
-    THANOS_CHECK_LAUNCH();
+    THANOS_TRY(convert_to_f32(static_cast<const __nv_bfloat16*>(W_in), Wc, nel, stream));
   } else {
     Wc = static_cast<float*>(W_out);
     if (W_in != W_out)
@@ -505,8 +482,7 @@ thanos_status_t prune_layer_structured_impl(const void* W_in, void* W_out, uint8
                                      (long long)s * (long long)(c - n_out), (int)s);
   THANOS_CHECK_LAUNCH();
   if (need_wc) {
-    f32_to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(Wc, static_cast<__nv_bfloat16*>(W_out), nel);
-    THANOS_CHECK_LAUNCH();
+    THANOS_TRY(convert_to_bf16(Wc, static_cast<__nv_bfloat16*>(W_out), nel, stream));
   }
   return THANOS_OK;
 }

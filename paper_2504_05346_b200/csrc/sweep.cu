@@ -943,6 +943,19 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
 
 }  // namespace
 
+// dtype conversion of a whole weight matrix (bf16 I/O <-> fp32 working copy)
+thanos_status_t convert_to_f32(const __nv_bfloat16* in, float* out, int64_t n, cudaStream_t stream) {
+  to_f32_kernel<<<148 * 8, 256, 0, stream>>>(in, out, n);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+thanos_status_t convert_to_bf16(const float* in, __nv_bfloat16* out, int64_t n, cudaStream_t stream) {
+  to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(in, out, n);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
 size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype) {
   size_t t = 0;
   const size_t blocks = (size_t)ceil_div(b, B);
@@ -1072,8 +1085,7 @@ thanos_status_t prune_layer_core(const void* W_in, void* W_out, uint8_t* mask_ou
   float* Wc;
   if (need_wc) {
     Wc = w.Wc;
-    to_f32_kernel<<<148 * 8, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(W_in), Wc, nel);
-    THANOS_CHECK_LAUNCH();
+    THANOS_TRY(convert_to_f32(static_cast<const __nv_bfloat16*>(W_in), Wc, nel, stream));
   } else {
     Wc = static_cast<float*>(W_out);
     if (W_in != W_out)
@@ -1144,8 +1156,7 @@ thanos_status_t prune_layer_core(const void* W_in, void* W_out, uint8_t* mask_ou
   fold_tc_status_kernel<<<1, 1, 0, stream>>>(stats, w.tc_status);
   THANOS_CHECK_LAUNCH();
   if (need_wc) {
-    to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(Wc, static_cast<__nv_bfloat16*>(W_out), nel);
-    THANOS_CHECK_LAUNCH();
+    THANOS_TRY(convert_to_bf16(Wc, static_cast<__nv_bfloat16*>(W_out), nel, stream));
   }
   return THANOS_OK;
 }
