@@ -61,7 +61,7 @@ __host__ __device__ inline SolveSmemLayout solve_layout(int Bw, int panels, bool
 // are split between the kinds in proportion to the list lengths; without them every row is of
 // kind `fixed_kind`.
 template <int NR>
-__global__ void __launch_bounds__(384)
+__global__ void __launch_bounds__(32 * 15)
 solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                        const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
                        __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw, int ldd,
@@ -412,6 +412,8 @@ solve_rows_fast_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
 }
 
 constexpr size_t SOLVE_SMEM_BUDGET = 227 * 1024;  // the most dynamic shared memory a CTA can get
+constexpr int SOLVE_MAX_WARPS = 15;               // launch bound of solve_rows_fast_kernel
+constexpr float UNCACHED_ROW_COST = 1.4f;         // time of a row without the shared copy of G / S over with it
 
 template <int NR>
 thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, const float* S,
@@ -420,11 +422,29 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
                             const int* row_lists, const unsigned* list_counts, int fixed_kind,
                             int report_max_s, thanos_stats_t* stats, cudaStream_t stream) {
   const int panels = (n_max + 1 + 7) / 8;
-  bool in_smem = (size_t)Bw * (Bw | 1) * 4 <= 72 * 1024;
-  SolveSmemLayout lay = solve_layout(Bw, panels, in_smem);
-  int warps = (int)((SOLVE_SMEM_BUDGET - 4 * (size_t)lay.mat_floats) / lay.per_warp_bytes);
+  // A warp works through its rows one after the other, and a row takes about the same time
+  // whatever else is resident on the SM: a launch lasts (rows per warp, rounded up) x (time of a
+  // row).  With G / S copied to shared memory a row is faster (33-35 us against 45-50 us at
+  // B = 128, 50 %), but the copy leaves room for fewer warps; take whichever comes out shorter.
+  const bool can_copy = (size_t)Bw * (Bw | 1) * 4 <= 72 * 1024;
+  bool in_smem = false;
+  int warps = 0;
+  float best = 0.f;
+  for (int copy = can_copy ? 1 : 0; copy >= 0; --copy) {
+    const SolveSmemLayout l = solve_layout(Bw, panels, copy != 0);
+    int wmax = (int)((SOLVE_SMEM_BUDGET - 4 * (size_t)l.mat_floats) / l.per_warp_bytes);
+    if (wmax > SOLVE_MAX_WARPS) wmax = SOLVE_MAX_WARPS;
+    for (int w = wmax; w >= 1 && w >= wmax - 1; --w) {
+      const float cost = (float)ceil_div(c, (int64_t)148 * w) * (copy ? 1.f : UNCACHED_ROW_COST);
+      if (warps == 0 || cost < best || (cost == best && copy == 0 && !in_smem)) {
+        best = cost;
+        warps = w;
+        in_smem = copy != 0;
+      }
+    }
+  }
   if (warps < 1) return THANOS_ERR_SHAPE;
-  if (warps > 12) warps = 12;
+  SolveSmemLayout lay = solve_layout(Bw, panels, in_smem);
   const size_t smem = 4 * (size_t)lay.mat_floats + (size_t)warps * lay.per_warp_bytes;
   {
     static std::atomic<unsigned long long> done{0};
