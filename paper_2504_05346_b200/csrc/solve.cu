@@ -490,7 +490,9 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
   const int* rl = uniform ? nullptr : row_lists;
   const unsigned* lc = uniform ? nullptr : list_counts;
   const int rep = uniform ? 1 : 0;
-  if (n_small + 1 > 160)
+  // 97 to 159 unknowns in a block of at most 256 columns: the four-warp CTAs of solve_cta.cu
+  // keep four rows per SM in flight, the warp-per-row kernel (41 KB per warp) only five warps
+  if (n_small + 1 > 160 || (n_small + 1 > 96 && Bw <= 256))
     return launch_cta_solve(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                             fixed_kind, rep, stats, stream);
   if (n_small + 1 <= 32)

@@ -1,12 +1,13 @@
 // Per-row constrained solve for large systems (Eqs. 5-8): one CTA per row.
 //
 // Same mathematics as the warp-per-row kernel (direct form on G for rows with |q| <= |k|,
-// complement form on S otherwise), for systems of 160 to 319 unknowns -- e.g. 2:4 sparsity with
-// the block width B = 512 of Section 5, where every row solves a 256 x 256 system.  The gathered
+// complement form on S otherwise), for systems of 97 to 319 unknowns -- e.g. 2:4 sparsity with
+// the block width B = 512 of Section 5, where every row solves a 256 x 256 system, or 4:8 with
+// B = 256 (128 unknowns).  The gathered
 // matrix lives in shared memory as the lower triangle of 16 x 16 tiles (1 KB each, 16-byte chunks
 // swizzled by the row so that the accesses below are free of bank conflicts); the right-hand
 // side is appended as row n, so that the factorisation L L^T also yields y = L^{-1} rhs.
-// Right-looking tile Cholesky by 8 warps: panel solve (one thread per row), trailing update
+// Right-looking tile Cholesky by the CTA's warps (16, or 4 for the smaller systems): panel solve (one thread per row), trailing update
 // (one warp per target tile, handed out by a shared counter); warp 0 updates and factors the
 // next diagonal tile first, which takes the only serial step off the critical path.  Blocked
 // back substitution L^T x = y, then the change of the block's weights as in the small kernel.
@@ -22,8 +23,6 @@ using tile::elem_off;
 using tile::tile_update;
 
 constexpr unsigned FULL = 0xffffffffu;
-constexpr int CTA_THREADS = 512;
-constexpr int CTA_WARPS = CTA_THREADS / 32;
 constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 - 1 = 319 unknowns
 
 // tile (I, J), J <= I, of the lower triangle; 256 floats each
@@ -97,7 +96,8 @@ __device__ __forceinline__ void macro_update(float* __restrict__ A, int K, int I
     }
 }
 
-// exclusive prefix sum of one value per thread over the CTA (256 threads)
+// exclusive prefix sum of one value per thread over the CTA
+template <int CTA_WARPS>
 __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* warp_sums,
                                                        unsigned& total) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -123,7 +123,13 @@ __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* war
 
 // Rows come from row_lists[2][c] / list_counts[2] (kind 0: |q| <= |k|, direct form on G; kind 1:
 // complement form on S), or are all rows with kind `fixed_kind` when row_lists is null.
-__global__ void __launch_bounds__(CTA_THREADS, 1)
+//
+// CTA_THREADS = 512: one CTA per SM, for the largest systems (the tiles of one row fill most of the
+// shared memory).  CTA_THREADS = 128: four CTAs per SM for systems of 96 to 159 unknowns, where
+// four rows in flight with four warps each beat both one row with sixteen warps and the
+// warp-per-row kernel (whose 41 KB per warp leave room for five rows per SM).
+template <int CTA_THREADS>
+__global__ void __launch_bounds__(CTA_THREADS, 512 / CTA_THREADS)
 solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                       const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
                       __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
@@ -171,7 +177,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       if (c1 < Bw) wblk[c1] = wrow[c1];
       const unsigned mine = (unsigned)((m0 == 1) + (m1 == 1)) | ((unsigned)((m0 == 0) + (m1 == 0)) << 16);
       unsigned all;
-      const unsigned before = cta_exclusive_scan(mine, warp_sums, all);
+      const unsigned before = cta_exclusive_scan<CTA_THREADS / 32>(mine, warp_sums, all);
       int pq = (int)(before & 0xffffu), pk = (int)(before >> 16);
       if (m0 == 1) qlist[pq++] = (unsigned short)c0;
       if (m0 == 0) klist[pk++] = (unsigned short)c0;
@@ -229,9 +235,12 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     __syncthreads();
     // ---- gather the lower triangle of M[sel, sel], the right-hand-side row n, identity padding
     {
-      // 256 threads fill one tile; the CTA's groups of 256 threads take tiles round-robin
-      constexpr int GROUPS = CTA_THREADS / 256;
-      const int r = (tid & 255) >> 4, k = tid & 15, grp = tid >> 8;
+      // A tile has 256 entries: with 512 threads two tiles are filled at a time, with 128 threads
+      // a thread fills two entries of each tile; eight tiles' loads are in flight per thread.
+      constexpr int GROUPS = CTA_THREADS >= 256 ? CTA_THREADS / 256 : 1;  // tiles at a time
+      constexpr int PER = CTA_THREADS >= 256 ? 1 : 256 / CTA_THREADS;     // entries per thread and tile
+      constexpr int RSTEP = CTA_THREADS >= 256 ? 16 : CTA_THREADS / 16;   // row step between them
+      const int r0 = (tid & 255) >> 4, k = tid & 15, grp = tid >> 8;
       const int ntiles = (T * (T + 1)) >> 1;
       int I = 0, J = 0;
       for (int g = 0; g < grp; ++g)
@@ -239,21 +248,25 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           ++I;
           J = 0;
         }
-      for (int t0 = grp; t0 < ntiles; t0 += 8 * GROUPS) {  // eight loads in flight per thread
-        float v[8];
+      for (int t0 = grp; t0 < ntiles; t0 += 8 * GROUPS) {
+        float v[8][PER];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-          const int i = 16 * I + r, j = 16 * J + k;
-          float x;
-          if (t0 + u * GROUPS >= ntiles)
-            x = 0.f;
-          else if (i < n)
-            x = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
-          else if (i == n)
-            x = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
-          else
-            x = i == j ? 1.f : 0.f;
-          v[u] = x;
+#pragma unroll
+          for (int h = 0; h < PER; ++h) {
+            const int r = r0 + RSTEP * h;
+            const int i = 16 * I + r, j = 16 * J + k;
+            float x;
+            if (t0 + u * GROUPS >= ntiles)
+              x = 0.f;
+            else if (i < n)
+              x = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
+            else if (i == n)
+              x = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
+            else
+              x = i == j ? 1.f : 0.f;
+            v[u][h] = x;
+          }
 #pragma unroll
           for (int g = 0; g < GROUPS; ++g)
             if (++J > I) {
@@ -263,7 +276,10 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-          if (t0 + u * GROUPS < ntiles) A[((t0 + u * GROUPS) << 8) + elem_off(r, k)] = v[u];
+#pragma unroll
+          for (int h = 0; h < PER; ++h)
+            if (t0 + u * GROUPS < ntiles)
+              A[((t0 + u * GROUPS) << 8) + elem_off(r0 + RSTEP * h, k)] = v[u][h];
       }
     }
     __syncthreads();
@@ -396,25 +412,41 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
 // Largest system (unknowns) the CTA-per-row kernel holds.
 int cta_solve_max_unknowns() { return 16 * MAX_TILES - 1; }
 
+template <int CTA_THREADS>
+thanos_status_t launch_cta_solve_t(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                   int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b,
+                                   int j1, int Bw, int ldd, int tiles, size_t smem,
+                                   const int* row_lists, const unsigned* list_counts,
+                                   int fixed_kind, int report_max_s, thanos_stats_t* stats,
+                                   cudaStream_t stream) {
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_cta_kernel<CTA_THREADS>, 227 * 1024, done));
+  }
+  const int ctas = 148 * (512 / CTA_THREADS);
+  const int grid = c < ctas ? c : ctas;
+  solve_rows_cta_kernel<CTA_THREADS><<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
+      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,
+      fixed_kind, report_max_s, stats);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
 thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
                                  int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
                                  int Bw, int ldd, int n_max, const int* row_lists,
                                  const unsigned* list_counts, int fixed_kind, int report_max_s,
                                  thanos_stats_t* stats, cudaStream_t stream) {
   const int tiles = (n_max + 16) / 16;
-  if (tiles > MAX_TILES || Bw > 2 * CTA_THREADS) return THANOS_ERR_SHAPE;
+  if (tiles > MAX_TILES || Bw > 1024) return THANOS_ERR_SHAPE;
   const size_t smem = cta_smem_bytes(tiles, Bw);
   if (smem > 227 * 1024) return THANOS_ERR_SHAPE;
-  {
-    static std::atomic<unsigned long long> done{0};
-    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_cta_kernel, 227 * 1024, done));
-  }
-  int grid = c < 148 ? c : 148;
-  solve_rows_cta_kernel<<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
-      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,
-      fixed_kind, report_max_s, stats);
-  THANOS_CHECK_LAUNCH();
-  return THANOS_OK;
+  // small tile sets: four CTAs of four warps per SM (a thread owns two columns of the block)
+  if (smem <= 56 * 1024 && Bw <= 256)
+    return launch_cta_solve_t<128>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, smem,
+                                   row_lists, list_counts, fixed_kind, report_max_s, stats, stream);
+  return launch_cta_solve_t<512>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, smem,
+                                 row_lists, list_counts, fixed_kind, report_max_s, stats, stream);
 }
 
 }  // namespace thanos
