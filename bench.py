@@ -74,7 +74,40 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
 
+    def _nvml_loop(self):
+        import pynvml as N
+        names = [("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap")]
+        bits = [(nm, getattr(N, const)) for nm, const in names if hasattr(N, const)]
+        while not self._stop.is_set():
+            try:
+                self._sm.append(float(N.nvmlDeviceGetClockInfo(self._h, N.NVML_CLOCK_SM)))
+                r = int(N.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for nm, bit in bits:
+                    if r & bit:
+                        self._reasons.add(nm)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
     def start(self):
+        """Read-only NVML queries every 20 ms from a thread; nvidia-smi (200 ms) if NVML is not
+        importable."""
+        import threading
+        self._sm, self._reasons, self._thread = [], set(), None
+        try:
+            import pynvml as N
+            N.nvmlInit()
+            self._h = N.nvmlDeviceGetHandleByIndex(self.gpu)
+            self._smax = float(N.nvmlDeviceGetMaxClockInfo(self._h, N.NVML_CLOCK_SM))
+            self._stop = threading.Event()
+            self._thread = threading.Thread(target=self._nvml_loop, daemon=True)
+            self._thread.start()
+            return
+        except Exception:
+            self._thread = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
@@ -84,6 +117,12 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
+        if getattr(self, "_thread", None) is not None:
+            self._stop.set()
+            self._thread.join(timeout=2)
+            sm = self._sm
+            return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self._smax,
+                    "samples": len(sm), "reasons": sorted(self._reasons)}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
