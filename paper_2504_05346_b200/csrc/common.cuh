@@ -47,6 +47,9 @@ inline cudaError_t ensure_max_dyn_smem(F func, int bytes, std::atomic<unsigned l
   return e;
 }
 
+// Grids are sized for the 148 SMs of a B200 (this library is built for sm_100a only).
+constexpr int NUM_SMS = 148;
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

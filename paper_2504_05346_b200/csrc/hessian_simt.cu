@@ -59,7 +59,7 @@ thanos_status_t hessian_accumulate_simt(float* H, int64_t b, const void* X, than
   int nt = (int)ceil_div(b, HB);
   int npairs = nt * (nt + 1) / 2;
   // slice tokens so the grid has a few waves of CTAs; each slice is at most 2^30 tokens
-  int64_t want_slices = ceil_div(148 * 4, npairs);
+  int64_t want_slices = ceil_div(NUM_SMS * 4, npairs);
   int64_t tok_per_slice = ceil_div(n_tok, want_slices);
   tok_per_slice = round_up((size_t)(tok_per_slice < 256 ? 256 : tok_per_slice), HK);
   if (tok_per_slice > (1 << 30)) tok_per_slice = 1 << 30;

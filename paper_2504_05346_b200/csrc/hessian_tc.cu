@@ -430,7 +430,7 @@ thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos
   __nv_bfloat16* planes = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + 256);
   for (int64_t t0 = 0; t0 < n_tok; t0 += SPLIT_CHUNK) {
     int n = (int)(n_tok - t0 < SPLIT_CHUNK ? n_tok - t0 : SPLIT_CHUNK);
-    split_planes_kernel<<<148 * 8, 256, 0, stream>>>(static_cast<const float*>(X) + t0 * ldx, ldx,
+    split_planes_kernel<<<NUM_SMS * 8, 256, 0, stream>>>(static_cast<const float*>(X) + t0 * ldx, ldx,
                                                      n, (int)b, planes);
     THANOS_CHECK_LAUNCH();
     THANOS_TRY(launch_tc(H, (int)b, planes, b, n, 3, (int64_t)n * b, status, stream));

@@ -435,7 +435,7 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
     int wmax = (int)((SOLVE_SMEM_BUDGET - 4 * (size_t)l.mat_floats) / l.per_warp_bytes);
     if (wmax > SOLVE_MAX_WARPS) wmax = SOLVE_MAX_WARPS;
     for (int w = wmax; w >= 1 && w >= wmax - 1; --w) {
-      const float cost = (float)ceil_div(c, (int64_t)148 * w) * (copy ? 1.f : UNCACHED_ROW_COST);
+      const float cost = (float)ceil_div(c, (int64_t)NUM_SMS * w) * (copy ? 1.f : UNCACHED_ROW_COST);
       if (warps == 0 || cost < best || (cost == best && copy == 0 && !in_smem)) {
         best = cost;
         warps = w;
@@ -451,7 +451,7 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
     THANOS_CUDA(ensure_max_dyn_smem(solve_rows_fast_kernel<NR>, (int)SOLVE_SMEM_BUDGET, done));
   }
   int64_t grid = ceil_div(c, warps);
-  if (grid > 148) grid = 148;
+  if (grid > NUM_SMS) grid = NUM_SMS;
   solve_rows_fast_kernel<NR><<<(unsigned)grid, warps * 32, smem, stream>>>(
       Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, panels, in_smem ? 1 : 0, row_lists,
       list_counts, fixed_kind, report_max_s, stats);

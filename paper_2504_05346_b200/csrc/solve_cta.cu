@@ -423,7 +423,7 @@ thanos_status_t launch_cta_solve_t(float* Wc, const uint8_t* mask, const float* 
     static std::atomic<unsigned long long> done{0};
     THANOS_CUDA(ensure_max_dyn_smem(solve_rows_cta_kernel<CTA_THREADS>, 227 * 1024, done));
   }
-  const int ctas = 148 * (512 / CTA_THREADS);
+  const int ctas = NUM_SMS * (512 / CTA_THREADS);
   const int grid = c < ctas ? c : ctas;
   solve_rows_cta_kernel<CTA_THREADS><<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
       Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,

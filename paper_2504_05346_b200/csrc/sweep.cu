@@ -888,12 +888,12 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    int hg = c < 148 * 8 ? c : 148 * 8;
+    int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
-    const int sg = c < 148 * 4 ? c : 148 * 4;
+    const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
     for (int pass = 0; pass < 5; ++pass) {
       // passes after the first usually look at the copied keys only, or do nothing
-      const int sgp = pass == 0 ? sg : (sg < 148 * 2 ? sg : 148 * 2);
+      const int sgp = pass == 0 ? sg : (sg < NUM_SMS * 2 ? sg : NUM_SMS * 2);
       select_pass_kernel<<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
                                                  w.list_counts, pass == 0 ? 1 : 0, stats, w.cand,
                                                  (unsigned)w.cand_cap);
@@ -904,7 +904,7 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     tie_scan_kernel<<<1, 1024, 0, stream>>>(c, w.st, w.rowcnt, w.rowbase);
     THANOS_CHECK_LAUNCH();
     int mg = (int)ceil_div(c, 8);
-    if (mg > 148 * 8) mg = 148 * 8;
+    if (mg > NUM_SMS * 8) mg = NUM_SMS * 8;
     mark_block_kernel<<<mg, 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
                                               w.row_lists, w.list_counts, stats, r_ext);
     THANOS_CHECK_LAUNCH();
@@ -945,13 +945,13 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
 
 // dtype conversion of a whole weight matrix (bf16 I/O <-> fp32 working copy)
 thanos_status_t convert_to_f32(const __nv_bfloat16* in, float* out, int64_t n, cudaStream_t stream) {
-  to_f32_kernel<<<148 * 8, 256, 0, stream>>>(in, out, n);
+  to_f32_kernel<<<NUM_SMS * 8, 256, 0, stream>>>(in, out, n);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
 
 thanos_status_t convert_to_bf16(const float* in, __nv_bfloat16* out, int64_t n, cudaStream_t stream) {
-  to_bf16_kernel<<<148 * 8, 256, 0, stream>>>(in, out, n);
+  to_bf16_kernel<<<NUM_SMS * 8, 256, 0, stream>>>(in, out, n);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }

@@ -503,7 +503,7 @@ thanos_status_t split3_planes(const float* X, int64_t ld, int64_t rows, int64_t 
   if (rows <= 0 || cols <= 0) return THANOS_OK;
   if (cols % 4 || ld % 4 || ldp % 4 || plane_stride % 4) return THANOS_ERR_ALIGNMENT;
   int64_t blocks = ceil_div(rows * (cols / 4), 256);
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > NUM_SMS * 16) blocks = NUM_SMS * 16;
   split3_kernel<<<(unsigned)blocks, 256, 0, stream>>>(X, ld, rows, cols, planes, ldp, plane_stride);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
