@@ -30,8 +30,8 @@ namespace {
 // the running budget r of Algorithm 1).  Keys are the fp32 bit patterns of |w| * ||X_j|| (>= 0, so
 // they order like the values).  Two routes, both exact:
 //   bracket  the threshold moves little from block to block, so one pass counts the keys below a
-//            window of 2^18 key values around the previous threshold, bins the keys inside it
-//            (512 bins of 512 values) and copies them out (about 3 in 100); a second, short pass
+//            window of 2^16 key values around the previous threshold, bins the keys inside it
+//            (512 bins of 128 values) and copies them out (about 1 in 130); a second, short pass
 //            over the copied keys resolves the 512 values of the hit bin;
 //   radix    four passes over 8, 8, 8 and 7 key bits (first block, or when the window misses).
 // One kernel, launched five times per block, does whichever pass the sweep state asks for; the
@@ -39,8 +39,8 @@ namespace {
 constexpr int HIST_BINS = 512;
 constexpr int RADIX_BINS = 256;
 constexpr int RADIX_REPL = 8;           // shared-memory copies of a radix histogram (by lane & 7)
-constexpr unsigned WINDOW = 1u << 18;   // key values covered by the bracket
-constexpr int WINDOW_SHIFT = 9;         // 512 values per bracket bin
+constexpr unsigned WINDOW = 1u << 16;   // key values covered by the bracket (0.8 % of a binade)
+constexpr int WINDOW_SHIFT = 7;         // 128 values per bracket bin
 constexpr int CTA_CAND = 6144;          // keys inside the window one CTA can hold before copying out
 __host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0)); }
@@ -353,7 +353,7 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     }
   } else if (phase == PH_BRACKET) {
     // The hot pass: per element one multiply, one compare-and-count, one window test; keys inside
-    // the window (about 3 in 100) take the slow path that bins and copies them.
+    // the window (about 1 in 130) take the slow path that bins and copies them.
     const unsigned lo = st->lo;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
@@ -819,7 +819,7 @@ int lazy_group(int64_t b, int B) {
   return g < 1 ? 1 : (g > 8 ? 8 : g);
 }
 
-// room for one key in eight of the layer (the bracket window holds about three in a hundred)
+// room for one key in eight of the layer (the bracket window holds about one in 130)
 size_t cand_capacity(int64_t c, int64_t b) {
   size_t n = (size_t)c * (size_t)b / 8;
   if (n < 4096) n = 4096;
