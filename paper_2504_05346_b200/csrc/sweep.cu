@@ -39,8 +39,9 @@ namespace {
 constexpr int HIST_BINS = 512;
 constexpr int RADIX_BINS = 256;
 constexpr int RADIX_REPL = 8;           // shared-memory copies of a radix histogram (by lane & 7)
-constexpr unsigned WINDOW = 1u << 16;   // key values covered by the bracket (0.8 % of a binade)
-constexpr int WINDOW_SHIFT = 7;         // 128 values per bracket bin
+constexpr int WINDOW_LOG2 = 16;        // key values covered by the bracket: 2^16 (0.8 % of a binade),
+constexpr int WINDOW_LOG2_WIDE = 18;   // 2^18 for the rest of a sweep once a bracket has missed
+constexpr int WINDOW_BINS_LOG2 = 9;    // 512 bracket bins
 constexpr int CTA_CAND = 6144;          // keys inside the window one CTA can hold before copying out
 __host__ __device__ constexpr int pass_bits(int pass) { return pass == 3 ? 7 : 8; }
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 23 : (pass == 1 ? 15 : (pass == 2 ? 7 : 0)); }
@@ -68,7 +69,7 @@ struct SweepState {
   unsigned int mark_ticket;      // same for the mask kernel
   unsigned int cand_total;       // keys the bracket pass copied out of its window
   int cand_overflow;             // the copy did not fit: the refine pass rescans the residual
-  int pad;
+  int wide;                      // a bracket missed in this sweep: use the wide window
 };
 
 __device__ __forceinline__ unsigned metric_key(float w, float xn) {
@@ -355,6 +356,9 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     // The hot pass: per element one multiply, one compare-and-count, one window test; keys inside
     // the window (about 1 in 130) take the slow path that bins and copies them.
     const unsigned lo = st->lo;
+    const int wlog = st->wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2;
+    const unsigned WINDOW = 1u << wlog;
+    const int WINDOW_SHIFT = wlog - WINDOW_BINS_LOG2;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
 #pragma unroll 2
@@ -479,13 +483,14 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     if (k > bel) find_rank_bin(const_cast<const unsigned*>(vh), HIST_BINS, k - bel, bin, before, inbin);
     if (bin >= 0) {
       if (lane == 0) {
-        st->lo = vs->lo + ((unsigned)bin << WINDOW_SHIFT);
+        st->lo = vs->lo + ((unsigned)bin << ((vs->wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2) - WINDOW_BINS_LOG2));
         st->k_rem = k - bel - before;
       }
       next = PH_REFINE;
     } else {
       if (lane == 0) {
         st->prefix = 0;
+        st->wide = 1;
         stats->select_misses += 1;
       }
       next = PH_RADIX0;  // the window missed: full radix select, k_rem is still the rank
@@ -652,9 +657,10 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
   st->blk_count = 0;
   st->mark_ticket = 0;
   // next block: bracket around this threshold when there is one, else a full radix select
-  const bool bracket = !none && tau >= (WINDOW >> 1);
+  const unsigned half_window = 1u << ((vs->wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2) - 1);
+  const bool bracket = !none && tau >= half_window;
   st->have_prev = bracket ? 1 : 0;
-  st->lo = bracket ? tau - (WINDOW >> 1) : 0u;
+  st->lo = bracket ? tau - half_window : 0u;
   st->prefix = 0;
   st->phase = bracket ? PH_BRACKET : PH_RADIX0;
 }

@@ -741,3 +741,18 @@ def test_llama2_70b_width_8192_sampled_rows(T, mode):
     Wr = O.replay_rows(_np64(W)[rows], M.cpu().numpy()[rows], Hd, B)
     Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
     assert PU.rel_fro(_np64(Wp)[rows], Wr) <= PU.TOL_W_BF16
+
+
+def test_threshold_jumps_between_blocks(T):
+    """Column blocks of very different scale move the global threshold by far more than the
+    bracket window from one block to the next: the bracket misses, the radix passes take over
+    (and the window stays wide for the rest of the sweep); the result is still the oracle's."""
+    c, b, B = 96, 768, 64
+    W = WL.make_weight(c, b, "f32", seed=97)
+    g = torch.Generator().manual_seed(11)
+    blk_scale = torch.tensor([1.0, 30.0, 0.05, 8.0, 0.3, 100.0, 1.0, 0.01, 3.0, 50.0, 0.2, 5.0])
+    W = W * blk_scale.repeat_interleave(B)[None, :]
+    Xt = WL.make_activations(4096, b, "f32", "normal", 0.0, 0, 1.0, 23, 0, mix=0.4)
+    H = _gpu_hessian(T, Xt)
+    out = _check_sweep(T, W, H, "unstructured", 0.5, 0, 0, B, 0.01, PU.TOL_W_F32)
+    assert out["stats"].select_misses >= 1
