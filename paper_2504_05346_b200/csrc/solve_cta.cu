@@ -7,7 +7,8 @@
 // matrix lives in shared memory as the lower triangle of 16 x 16 tiles (1 KB each, 16-byte chunks
 // swizzled by the row so that the accesses below are free of bank conflicts); the right-hand
 // side is appended as row n, so that the factorisation L L^T also yields y = L^{-1} rhs.
-// Right-looking tile Cholesky by the CTA's warps (16, or 4 for the smaller systems): panel solve (one thread per row), trailing update
+// Right-looking tile Cholesky by the CTA's warps (16, or 4 for the smaller systems; with 16 warps
+// the trailing update runs on the tensor cores from bf16 planes of the panel, see below): panel solve (one thread per row), trailing update
 // (one warp per target tile, handed out by a shared counter); warp 0 updates and factors the
 // next diagonal tile first, which takes the only serial step off the critical path.  Blocked
 // back substitution L^T x = y, then the change of the block's weights as in the small kernel.
@@ -96,6 +97,104 @@ __device__ __forceinline__ void macro_update(float* __restrict__ A, int K, int I
     }
 }
 
+// ---- trailing update on the tensor cores: the rows of the current panel are kept a second time
+// as three bf16 planes (x = h + m + l, 24 significant bits; row stride 24 elements, which makes
+// the fragment loads below free of bank conflicts), and C_IJ -= L_IK L_JK^T is the sum of the six
+// plane products hh, hm, mh, hl, lh, mm by mma.sync m16n8k16 with fp32 accumulation.
+constexpr int PLANE_LD = 24;
+
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&d)[4], const uint32_t (&a)[4],
+                                                  const uint32_t (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// planes of one solved panel row (16 values read back from its tile)
+__device__ __forceinline__ void store_row_planes(const float* __restrict__ tile_row_src, int r,
+                                                 __nv_bfloat16* __restrict__ prow, int plane_stride) {
+  float x[16];
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+    const float4 v = *reinterpret_cast<const float4*>(tile_row_src + tile::chunk_off(r, cc));
+    x[4 * cc] = v.x; x[4 * cc + 1] = v.y; x[4 * cc + 2] = v.z; x[4 * cc + 3] = v.w;
+  }
+#pragma unroll
+  for (int pl = 0; pl < 3; ++pl) {
+    uint32_t w[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      // two values per conversion; the low half of the word is the lower column
+      const __nv_bfloat162 pr = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
+      w[e] = *reinterpret_cast<const uint32_t*>(&pr);
+      if (pl < 2) {
+        x[2 * e] -= __uint_as_float(w[e] << 16);
+        x[2 * e + 1] -= __uint_as_float(w[e] & 0xffff0000u);
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(prow + (size_t)pl * plane_stride);
+    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  }
+}
+
+// 2 x 2 target tiles (I0 + di, J0 + dj) of step K from the panel's planes.  pa / pb: first panel
+// row of the tiles I0 / J0.  Fragment layout of mma.m16n8k16 (g = lane / 4, t = lane % 4):
+// A: rows g, g + 8, columns 2t, 2t + 1 (+8);  B: column g of the 8, rows (= k) 2t, 2t + 1 (+8);
+// C: rows g, g + 8, columns 2t, 2t + 1 of the 8.
+__device__ __forceinline__ void macro_update_mma(float* __restrict__ A, int K, int I0, int J0, int T,
+                                                 unsigned vmask, const __nv_bfloat16* __restrict__ Pp,
+                                                 int plane_stride, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  const int m = T - K - 1;  // tile rows in the panel
+  uint32_t af[2][3][4], bf[2][3][2][2];
+#pragma unroll
+  for (int d = 0; d < 2; ++d) {
+    const int ti = min(I0 - K - 1 + d, m - 1), tj = min(J0 - K - 1 + d, m - 1);  // clamped loads
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      const __nv_bfloat16* pa = Pp + (size_t)pl * plane_stride + (size_t)(16 * ti) * PLANE_LD;
+      const __nv_bfloat16* pb = Pp + (size_t)pl * plane_stride + (size_t)(16 * tj) * PLANE_LD;
+      af[d][pl][0] = *reinterpret_cast<const uint32_t*>(pa + g * PLANE_LD + 2 * t);
+      af[d][pl][1] = *reinterpret_cast<const uint32_t*>(pa + (g + 8) * PLANE_LD + 2 * t);
+      af[d][pl][2] = *reinterpret_cast<const uint32_t*>(pa + g * PLANE_LD + 2 * t + 8);
+      af[d][pl][3] = *reinterpret_cast<const uint32_t*>(pa + (g + 8) * PLANE_LD + 2 * t + 8);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        bf[d][pl][h][0] = *reinterpret_cast<const uint32_t*>(pb + (8 * h + g) * PLANE_LD + 2 * t);
+        bf[d][pl][h][1] = *reinterpret_cast<const uint32_t*>(pb + (8 * h + g) * PLANE_LD + 2 * t + 8);
+      }
+    }
+  }
+#pragma unroll
+  for (int di = 0; di < 2; ++di)
+#pragma unroll
+    for (int dj = 0; dj < 2; ++dj) {
+      if (!(vmask & (1u << (2 * di + dj)))) continue;  // warp-uniform
+      float* Ct = A + tile_base(I0 + di, J0 + dj);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        // smallest products first
+        mma_bf16_m16n8k16(acc, af[di][1], bf[dj][1][h]);  // m m
+        mma_bf16_m16n8k16(acc, af[di][2], bf[dj][0][h]);  // l h
+        mma_bf16_m16n8k16(acc, af[di][0], bf[dj][2][h]);  // h l
+        mma_bf16_m16n8k16(acc, af[di][1], bf[dj][0][h]);  // m h
+        mma_bf16_m16n8k16(acc, af[di][0], bf[dj][1][h]);  // h m
+        mma_bf16_m16n8k16(acc, af[di][0], bf[dj][0][h]);  // h h
+        float2* c0 = reinterpret_cast<float2*>(Ct + tile::elem_off(g, 8 * h + 2 * t));
+        float2* c1 = reinterpret_cast<float2*>(Ct + tile::elem_off(g + 8, 8 * h + 2 * t));
+        float2 v0 = *c0, v1 = *c1;
+        v0.x -= acc[0]; v0.y -= acc[1];
+        v1.x -= acc[2]; v1.y -= acc[3];
+        *c0 = v0;
+        *c1 = v1;
+      }
+    }
+}
+
 // exclusive prefix sum of one value per thread over the CTA
 template <int CTA_WARPS>
 __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* warp_sums,
@@ -135,7 +234,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                       __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
                       int ldd, int tiles, const int* __restrict__ row_lists,
                       const unsigned* __restrict__ list_counts, int fixed_kind, int report_max_s,
-                      thanos_stats_t* stats) {
+                      int use_planes, thanos_stats_t* stats) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -152,6 +251,10 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   unsigned* warp_sums = scratch;          // [32]
   unsigned* s_counter = scratch + 32;
   unsigned* s_bad = scratch + 33;
+  // planes of the current panel (tensor-core trailing update), 16-byte aligned behind the scratch
+  __nv_bfloat16* Pp = reinterpret_cast<__nv_bfloat16*>(
+      dyn + ((reinterpret_cast<unsigned char*>(scratch + 48) - dyn + 15) & ~(size_t)15));
+  const int plane_stride = 16 * (tiles - 1) * PLANE_LD;
 
   int cnt0, cnt1;
   if (row_lists) {
@@ -296,6 +399,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         for (int ii = tid; ii < 16 * m; ii += CTA_THREADS) {
           const int I = K + 1 + (ii >> 4), r = ii & 15;
           tile::panel_row_solve(A + tile_base(I, K), r, Lk, invd + 16 * K);
+          if (use_planes) store_row_planes(A + tile_base(I, K), r, Pp + (size_t)ii * PLANE_LD, plane_stride);
         }
       }
       __syncthreads();
@@ -331,7 +435,12 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
               const int I = I0 + di, J = J0 + dj;
               if (I < T && J <= I && J < Tf && !(I == K + 1 && J == K + 1)) vmask |= 1u << (2 * di + dj);
             }
-          if (vmask) macro_update(A, K, I0, J0, T, vmask, lane);
+          if (vmask) {
+            if (use_planes)
+              macro_update_mma(A, K, I0, J0, T, vmask, Pp, plane_stride, lane);
+            else
+              macro_update(A, K, I0, J0, T, vmask, lane);
+          }
         }
       }
       __syncthreads();
@@ -415,7 +524,7 @@ int cta_solve_max_unknowns() { return 16 * MAX_TILES - 1; }
 template <int CTA_THREADS>
 thanos_status_t launch_cta_solve_t(float* Wc, const uint8_t* mask, const float* G, const float* S,
                                    int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b,
-                                   int j1, int Bw, int ldd, int tiles, size_t smem,
+                                   int j1, int Bw, int ldd, int tiles, size_t smem, int use_planes,
                                    const int* row_lists, const unsigned* list_counts,
                                    int fixed_kind, int report_max_s, thanos_stats_t* stats,
                                    cudaStream_t stream) {
@@ -427,7 +536,7 @@ thanos_status_t launch_cta_solve_t(float* Wc, const uint8_t* mask, const float* 
   const int grid = c < ctas ? c : ctas;
   solve_rows_cta_kernel<CTA_THREADS><<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
       Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,
-      fixed_kind, report_max_s, stats);
+      fixed_kind, report_max_s, use_planes, stats);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
@@ -443,9 +552,13 @@ thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G,
   if (smem > 227 * 1024) return THANOS_ERR_SHAPE;
   // small tile sets: four CTAs of four warps per SM (a thread owns two columns of the block)
   if (smem <= 56 * 1024 && Bw <= 256)
-    return launch_cta_solve_t<128>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, smem,
+    return launch_cta_solve_t<128>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, smem, 0,
                                    row_lists, list_counts, fixed_kind, report_max_s, stats, stream);
-  return launch_cta_solve_t<512>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, smem,
+  // the planes of a panel (tensor-core trailing update) when they still fit next to the tiles
+  const size_t with_planes = ((smem + 15) & ~(size_t)15) + 3 * (size_t)16 * (tiles - 1) * PLANE_LD * 2;
+  const int use_planes = with_planes <= 227 * 1024 ? 1 : 0;
+  return launch_cta_solve_t<512>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles,
+                                 use_planes ? with_planes : smem, use_planes,
                                  row_lists, list_counts, fixed_kind, report_max_s, stats, stream);
 }
 
