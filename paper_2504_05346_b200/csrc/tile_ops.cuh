@@ -10,8 +10,10 @@ namespace tile {
 constexpr unsigned FULL_MASK = 0xffffffffu;
 
 // A tile is 256 floats, row-major in 16-byte chunks; chunk c of row r sits at chunk position
-// c ^ ((r >> 1) & 3), which keeps the access patterns of the functions below free of bank conflicts.
-__device__ __forceinline__ int chunk_off(int r, int c) { return (r << 4) + (((c ^ (r >> 1)) & 3) << 2); }
+// c ^ swizzle(r) with swizzle = (bit 1 of r, bit 2 of r), which keeps the access patterns of the
+// functions below, and the accumulator fragments of mma.m16n8k16, free of bank conflicts.
+__device__ __forceinline__ int chunk_swizzle(int r) { return (r & 2) | ((r >> 2) & 1); }
+__device__ __forceinline__ int chunk_off(int r, int c) { return (r << 4) + ((c ^ chunk_swizzle(r)) << 2); }
 __device__ __forceinline__ int elem_off(int r, int k) { return chunk_off(r, k >> 2) + (k & 3); }
 
 // Cholesky of a diagonal tile by one warp: lane r < 16 holds row r.  Columns col0 + j >= n (a
