@@ -72,7 +72,10 @@ typedef struct {
   uint32_t last_threshold_bits; /* fp32 bit pattern of the last block's threshold metric  */
   int32_t select_misses; /* unstructured: blocks whose threshold fell outside the bracket around
                             the previous block's (they take the four-pass route)              */
-  int32_t reserved[4];
+  int32_t select_rescans; /* unstructured: blocks whose bracket held more keys than the copy-out
+                             buffers take (one CTA's share or the whole list), so that the
+                             refining pass read the residual a second time                     */
+  int32_t reserved[3];
 } thanos_stats_t;
 
 /*
@@ -209,7 +212,11 @@ size_t thanos_structured_workspace_bytes(int64_t c, int64_t b, double p, double 
  *  mask     device uint8 [c, b]; columns [j1, min(b, j1+B)) are written.
  *  r_dev    device int64: removals still to place (unstructured); read and decremented by the
  *           number of entries this block removed.  Ignored in NM mode (may be NULL).
- *  stats_dev is accumulated into, not zeroed.
+ *  stats_dev is accumulated into, not zeroed.  When it carries the statistics of the previous
+ *           block step of the same sweep (n_blocks > 0), the unstructured threshold search starts
+ *           from the bracket around last_threshold_bits (wide once select_misses > 0), exactly as
+ *           inside thanos_prune_layer; with a zeroed stats_dev it starts from scratch (four radix
+ *           passes).  Both routes give the same exact threshold.
  *  j1 % B == 0.  Same workspace as thanos_prune_layer.
  */
 thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t b,
@@ -229,6 +236,11 @@ thanos_status_t thanos_prune_block(float* Wc, uint8_t* mask, int64_t c, int64_t 
  *  holding H, the factor, the staged inputs and the per-call workspaces.
  *  If reuse_factor != 0 the Hessian and factor left in `arena` by the previous call with the
  *  same b are reused and X_host is not read (layers that share an input, e.g. q/k/v).
+ *  Unlike the device-pointer calls this one owns short-lived runtime objects: for the duration of
+ *  a call that reads X_host it creates one copy stream and five events (so that the copy of a
+ *  token chunk overlaps the accumulation of the previous one) and destroys them before returning;
+ *  it allocates no memory.  stats_host->status also reports a bounded wait that ran out inside the
+ *  Hessian accumulation (err_index -1) and a failed factorisation (err_index = column).
  */
 thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_host,
                                         void* W_out_host, uint8_t* mask_out_host,
@@ -260,6 +272,9 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
  * on a device share the one array: the call clears the parts that must start from zero, so
  * leftovers of an earlier call are harmless, but two calls that overlap on the GPU (different
  * streams, or different host threads) race on it -- serialise them.
+ *
+ * The array that is used is the current device's: make the device that holds W_in current
+ * before the call (weights on another device are refused with THANOS_ERR_INVALID_ARG).
  *
  * Arguments, layouts, results and device-side error reporting are those of
  * thanos_prune_layer, minus `workspace` and `ws_bytes`.

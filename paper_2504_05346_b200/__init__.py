@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     lib_path,
     load_library,
     hessian_accumulate,
+    hessian_status,
     prepare_inverse,
     prune_layer,
     prune_block,

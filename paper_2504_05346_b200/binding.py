@@ -33,7 +33,8 @@ class _Stats(ctypes.Structure):
         ("n_tied", ctypes.c_int64),
         ("last_threshold_bits", ctypes.c_uint32),
         ("select_misses", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 4),
+        ("select_rescans", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 3),
     ]
 
 
@@ -51,12 +52,13 @@ class PruneStats:
     n_tied: int
     last_threshold_bits: int
     select_misses: int = 0
+    select_rescans: int = 0
 
     @staticmethod
     def from_bytes(raw: bytes) -> "PruneStats":
         s = _Stats.from_buffer_copy(raw)
         return PruneStats(s.status, s.err_index, s.n_pruned, s.r_left, s.max_s, s.n_blocks,
-                          s.n_tied, s.last_threshold_bits, s.select_misses)
+                          s.n_tied, s.last_threshold_bits, s.select_misses, s.select_rescans)
 
 
 _lib = None
@@ -165,9 +167,23 @@ def _check(code: int, where: str):
         raise ThanosError(code, where)
 
 
+def _on(t: torch.Tensor):
+    """Makes the tensor's device current for the duration of a library call (kernels are
+    launched on, and per-device state is looked up for, the current device)."""
+    return torch.cuda.device(t.device)
+
+
+def hessian_status(workspace: torch.Tensor) -> int:
+    """Device status word of the last thanos_hessian_accumulate call that used `workspace`
+    (synchronises): 0, or THANOS_ERR_TIMEOUT (7) if a bounded wait inside the kernel ran out."""
+    return int(workspace[:4].view(torch.int32).item())
+
+
 def hessian_accumulate(H: torch.Tensor, X: torch.Tensor, stream=None,
-                       workspace: Optional[torch.Tensor] = None) -> None:
-    """H += 2 X^T X for tokens-major X [n_tok, b] (float32 or bfloat16); H float32 [b, b]."""
+                       workspace: Optional[torch.Tensor] = None, check: bool = False) -> None:
+    """H += 2 X^T X for tokens-major X [n_tok, b] (float32 or bfloat16); H float32 [b, b].
+    With check=True the call's device status word is read back (this waits for the call) and a
+    non-zero status raises."""
     lib = load_library()
     if not X.is_cuda or X.stride(-1) != 1:
         raise ValueError("X must be a CUDA tensor with unit inner stride")
@@ -178,9 +194,14 @@ def hessian_accumulate(H: torch.Tensor, X: torch.Tensor, stream=None,
     dt = _dtype_code(X)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_HESSIAN, 0, b, 0, dt), H.device)
-    _check(lib.thanos_hessian_accumulate(H.data_ptr(), b, X.data_ptr(), dt, n_tok, ldx,
-                                         workspace.data_ptr(), workspace.numel(),
-                                         _stream_ptr(stream)), "thanos_hessian_accumulate")
+    with _on(H):
+        _check(lib.thanos_hessian_accumulate(H.data_ptr(), b, X.data_ptr(), dt, n_tok, ldx,
+                                             workspace.data_ptr(), workspace.numel(),
+                                             _stream_ptr(stream)), "thanos_hessian_accumulate")
+        if check and n_tok > 0:
+            st = hessian_status(workspace)
+            if st != 0:
+                raise ThanosError(st, "thanos_hessian_accumulate (device)")
 
 
 def prepare_inverse(H: torch.Tensor, damp_rel: float, stream=None,
@@ -200,10 +221,11 @@ def prepare_inverse(H: torch.Tensor, damp_rel: float, stream=None,
     status = torch.zeros(4, dtype=torch.int32, device=H.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_PREPARE, 0, b, 0, F32), H.device)
-    _check(lib.thanos_prepare_inverse(H.data_ptr(), b, float(damp_rel), factor.data_ptr(),
-                                      xnorm.data_ptr(), workspace.data_ptr(), workspace.numel(),
-                                      status.data_ptr(), _stream_ptr(stream)),
-           "thanos_prepare_inverse")
+    with _on(H):
+        _check(lib.thanos_prepare_inverse(H.data_ptr(), b, float(damp_rel), factor.data_ptr(),
+                                          xnorm.data_ptr(), workspace.data_ptr(),
+                                          workspace.numel(), status.data_ptr(),
+                                          _stream_ptr(stream)), "thanos_prepare_inverse")
     if check:
         st = status.cpu()
         if int(st[0]) != 0:
@@ -231,10 +253,11 @@ def prune_layer(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tensor, mode
     stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_PRUNE, c, b, B, dt), W.device)
-    _check(lib.thanos_prune_layer(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
-                                  factor.data_ptr(), xnorm.data_ptr(), mode, float(p), n, m, B,
-                                  workspace.data_ptr(), workspace.numel(), stats.data_ptr(),
-                                  _stream_ptr(stream)), "thanos_prune_layer")
+    with _on(W):
+        _check(lib.thanos_prune_layer(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
+                                      factor.data_ptr(), xnorm.data_ptr(), mode, float(p), n, m, B,
+                                      workspace.data_ptr(), workspace.numel(), stats.data_ptr(),
+                                      _stream_ptr(stream)), "thanos_prune_layer")
     if not read_stats:
         return out, mask, stats
     st = _read_stats(stats)
@@ -252,11 +275,12 @@ def prune_block(Wc: torch.Tensor, mask: torch.Tensor, factor: torch.Tensor, xnor
     c, b = Wc.shape
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_PRUNE, c, b, B, F32), Wc.device)
-    _check(lib.thanos_prune_block(Wc.data_ptr(), mask.data_ptr(), c, b, factor.data_ptr(),
-                                  xnorm.data_ptr(), mode, n, m, B, j1,
-                                  r.data_ptr() if r is not None else None,
-                                  workspace.data_ptr(), workspace.numel(), stats.data_ptr(),
-                                  _stream_ptr(stream)), "thanos_prune_block")
+    with _on(Wc):
+        _check(lib.thanos_prune_block(Wc.data_ptr(), mask.data_ptr(), c, b, factor.data_ptr(),
+                                      xnorm.data_ptr(), mode, n, m, B, j1,
+                                      r.data_ptr() if r is not None else None,
+                                      workspace.data_ptr(), workspace.numel(), stats.data_ptr(),
+                                      _stream_ptr(stream)), "thanos_prune_block")
 
 
 def prune_layer_host(W_host: torch.Tensor, X_host: Optional[torch.Tensor], damp_rel: float,
@@ -283,15 +307,18 @@ def prune_layer_host(W_host: torch.Tensor, X_host: Optional[torch.Tensor], damp_
     if arena is None:
         arena = _ws(workspace_bytes(WS_HOST_LAYER, c, b, B, dt), device)
     stats = _Stats()
-    _check(lib.thanos_prune_layer_host(W_host.data_ptr(),
-                                       X_host.data_ptr() if X_host is not None else None,
-                                       out.data_ptr(), mask.data_ptr(), dt, c, b, a,
-                                       float(damp_rel), mode, float(p), n, m, B,
-                                       1 if reuse_factor else 0, arena.data_ptr(), arena.numel(),
-                                       ctypes.byref(stats), _stream_ptr(stream)),
-           "thanos_prune_layer_host")
+    with _on(arena):
+        code = lib.thanos_prune_layer_host(W_host.data_ptr(),
+                                           X_host.data_ptr() if X_host is not None else None,
+                                           out.data_ptr(), mask.data_ptr(), dt, c, b, a,
+                                           float(damp_rel), mode, float(p), n, m, B,
+                                           1 if reuse_factor else 0, arena.data_ptr(),
+                                           arena.numel(), ctypes.byref(stats),
+                                           _stream_ptr(stream))
+    _check(code, "thanos_prune_layer_host")
     st = PruneStats(stats.status, stats.err_index, stats.n_pruned, stats.r_left, stats.max_s,
-                    stats.n_blocks, stats.n_tied, stats.last_threshold_bits)
+                    stats.n_blocks, stats.n_tied, stats.last_threshold_bits, stats.select_misses,
+                    stats.select_rescans)
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_host (index %d)" % st.err_index)
     return out, mask, st
@@ -299,10 +326,12 @@ def prune_layer_host(W_host: torch.Tensor, X_host: Optional[torch.Tensor], damp_
 
 def prune_layer_noalloc(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tensor, mode: int,
                         p: float = 0.0, n: int = 0, m: int = 0, B: int = 128, stream=None,
-                        out: Optional[torch.Tensor] = None, mask: Optional[torch.Tensor] = None):
+                        out: Optional[torch.Tensor] = None, mask: Optional[torch.Tensor] = None,
+                        stats: Optional[torch.Tensor] = None):
     """thanos_prune_layer_noalloc: the sweep with the library's built-in 4 MiB scratch, for
-    callers that cannot allocate a workspace.  Only the outputs are created here (pass `out`
-    and `mask` to avoid even that).  Calls on one device must not overlap."""
+    callers that cannot allocate a workspace.  Only the outputs are created here; pass `out`,
+    `mask` and `stats` (64 bytes, uint8) and this function creates no device tensor at all.
+    Calls on one device must not overlap."""
     lib = load_library()
     _check_dev(W, factor, xnorm)
     c, b = W.shape
@@ -311,11 +340,13 @@ def prune_layer_noalloc(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tens
         out = torch.empty_like(W)
     if mask is None:
         mask = torch.empty((c, b), dtype=torch.uint8, device=W.device)
-    stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
-    _check(lib.thanos_prune_layer_noalloc(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
-                                          factor.data_ptr(), xnorm.data_ptr(), mode, float(p), n,
-                                          m, B, stats.data_ptr(), _stream_ptr(stream)),
-           "thanos_prune_layer_noalloc")
+    if stats is None:
+        stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
+    with _on(W):
+        _check(lib.thanos_prune_layer_noalloc(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c,
+                                              b, factor.data_ptr(), xnorm.data_ptr(), mode,
+                                              float(p), n, m, B, stats.data_ptr(),
+                                              _stream_ptr(stream)), "thanos_prune_layer_noalloc")
     st = _read_stats(stats)
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_noalloc (row %d)" % st.err_index)
@@ -340,10 +371,11 @@ def dense_product(A: torch.Tensor, B: torch.Tensor, b_transposed: bool = False, 
     assert out.stride(1) == 1
     nbytes = lib.thanos_dense_product_workspace(M, N, K)
     ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=A.device)
-    _check(lib.thanos_dense_product(out.data_ptr(), out.stride(0), A.data_ptr(), A.stride(0),
-                                    B.data_ptr(), B.stride(0), 1 if b_transposed else 0, M, N, K,
-                                    float(alpha), 1 if accumulate else 0, ws.data_ptr(), nbytes,
-                                    _stream_ptr(stream)), "thanos_dense_product")
+    with _on(A):
+        _check(lib.thanos_dense_product(out.data_ptr(), out.stride(0), A.data_ptr(), A.stride(0),
+                                        B.data_ptr(), B.stride(0), 1 if b_transposed else 0, M, N, K,
+                                        float(alpha), 1 if accumulate else 0, ws.data_ptr(), nbytes,
+                                        _stream_ptr(stream)), "thanos_dense_product")
     if check:
         st = int(ws[:4].view(torch.int32).item())
         if st != 0:
@@ -369,11 +401,12 @@ def prune_layer_outliers(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Ten
     stats = torch.zeros(64, dtype=torch.uint8, device=W.device)
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_PRUNE_OUTLIERS, c, b, B, dt), W.device)
-    _check(lib.thanos_prune_layer_outliers(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
-                                           factor.data_ptr(), xnorm.data_ptr(), H.data_ptr(), n, m,
-                                           B, float(alpha), flags.data_ptr(), workspace.data_ptr(),
-                                           workspace.numel(), stats.data_ptr(),
-                                           _stream_ptr(stream)), "thanos_prune_layer_outliers")
+    with _on(W):
+        _check(lib.thanos_prune_layer_outliers(W.data_ptr(), out.data_ptr(), mask.data_ptr(), dt, c, b,
+                                               factor.data_ptr(), xnorm.data_ptr(), H.data_ptr(), n, m,
+                                               B, float(alpha), flags.data_ptr(), workspace.data_ptr(),
+                                               workspace.numel(), stats.data_ptr(),
+                                               _stream_ptr(stream)), "thanos_prune_layer_outliers")
     st = _read_stats(stats)
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_outliers (row %d)" % st.err_index)
@@ -405,13 +438,14 @@ def prune_layer_structured(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.T
         if need == 0:
             raise ThanosError(1, "thanos_structured_workspace_bytes rejected the arguments")
         workspace = _ws(need, W.device)
-    _check(lib.thanos_prune_layer_structured(W.data_ptr(), out.data_ptr(), colrm.data_ptr(),
-                                             flags.data_ptr(), dt, c, b, factor.data_ptr(),
-                                             xnorm.data_ptr(),
-                                             H.data_ptr() if H is not None else None, float(p),
-                                             float(alpha), workspace.data_ptr(), workspace.numel(),
-                                             stats.data_ptr(), _stream_ptr(stream)),
-           "thanos_prune_layer_structured")
+    with _on(W):
+        _check(lib.thanos_prune_layer_structured(W.data_ptr(), out.data_ptr(), colrm.data_ptr(),
+                                                 flags.data_ptr(), dt, c, b, factor.data_ptr(),
+                                                 xnorm.data_ptr(),
+                                                 H.data_ptr() if H is not None else None, float(p),
+                                                 float(alpha), workspace.data_ptr(), workspace.numel(),
+                                                 stats.data_ptr(), _stream_ptr(stream)),
+               "thanos_prune_layer_structured")
     st = _read_stats(stats)
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_structured (index %d)" % st.err_index)

@@ -44,7 +44,29 @@ thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_ou
                                  int32_t m, int32_t B, void* workspace, size_t ws_bytes,
                                  thanos_stats_t* stats, cudaStream_t stream);
 
+// Host-side argument checks shared by thanos_prune_layer and thanos_prune_layer_noalloc
+// (everything except the workspace).
+thanos_status_t check_prune_layer_args(const void* W_in, const void* W_out, const uint8_t* mask_out,
+                                       thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                       const float* factor, const float* xnorm, thanos_mode_t mode,
+                                       double p, int32_t n, int32_t m, int32_t B,
+                                       const thanos_stats_t* stats_dev) {
+  if (!W_in || !W_out || !mask_out || !factor || !xnorm || !stats_dev)
+    return THANOS_ERR_INVALID_ARG;
+  if (wdtype != THANOS_F32 && wdtype != THANOS_BF16) return THANOS_ERR_DTYPE;
+  THANOS_TRY(validate_sweep_args(c, b, mode, p, n, m, B));
+  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(mask_out) || !aligned16(factor) ||
+      !aligned16(xnorm) || !aligned16(stats_dev))
+    return THANOS_ERR_ALIGNMENT;
+  return THANOS_OK;
+}
+
 namespace {
+
+// dst keeps the first non-zero status word it is offered
+__global__ void fold_word_kernel(int32_t* dst, const int32_t* src) {
+  if (*src != 0 && *dst == 0) *dst = *src;
+}
 
 constexpr int64_t MAX_B = 65536;
 constexpr int64_t HOST_TOKEN_CHUNK = 16384;
@@ -123,13 +145,9 @@ thanos_status_t thanos_prune_layer(const void* W_in, void* W_out, uint8_t* mask_
                                    const float* factor, const float* xnorm, thanos_mode_t mode,
                                    double p, int32_t n, int32_t m, int32_t B, void* workspace,
                                    size_t ws_bytes, thanos_stats_t* stats_dev, void* stream) {
-  if (!W_in || !W_out || !mask_out || !factor || !xnorm || !stats_dev)
-    return THANOS_ERR_INVALID_ARG;
-  if (!dtype_ok(wdtype)) return THANOS_ERR_DTYPE;
-  THANOS_TRY(validate_sweep_args(c, b, mode, p, n, m, B));
-  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(mask_out) || !aligned16(factor) ||
-      !aligned16(xnorm) || !aligned16(workspace) || !aligned16(stats_dev))
-    return THANOS_ERR_ALIGNMENT;
+  THANOS_TRY(check_prune_layer_args(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, mode, p, n,
+                                    m, B, stats_dev));
+  if (!aligned16(workspace)) return THANOS_ERR_ALIGNMENT;
   if (!workspace || ws_bytes < prune_workspace_bytes(c, b, B, wdtype)) return THANOS_ERR_WORKSPACE;
   return prune_layer_impl(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, mode, p, n, m, B,
                           workspace, ws_bytes, stats_dev, static_cast<cudaStream_t>(stream));
@@ -240,40 +258,55 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
     THANOS_CUDA(cudaMemsetAsync(status, 0, 16, stream));
     // Two staging buffers: the copy of chunk k+1 is issued on a second stream while chunk k is
     // being accumulated.
-    cudaStream_t copy_stream;
-    cudaEvent_t copied[2], consumed[2];
-    THANOS_CUDA(cudaStreamCreateWithFlags(&copy_stream, cudaStreamNonBlocking));
-    for (int i = 0; i < 2; ++i) {
-      cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming);
-      cudaEventCreateWithFlags(&consumed[i], cudaEventDisableTiming);
-    }
-    cudaEvent_t start;
-    cudaEventCreateWithFlags(&start, cudaEventDisableTiming);
-    cudaEventRecord(start, stream);
-    cudaStreamWaitEvent(copy_stream, start, 0);
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t evs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     thanos_status_t st = THANOS_OK;
+    if (cudaStreamCreateWithFlags(&copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+      st = THANOS_ERR_CUDA;
+    for (int i = 0; i < 5 && st == THANOS_OK; ++i)
+      if (cudaEventCreateWithFlags(&evs[i], cudaEventDisableTiming) != cudaSuccess)
+        st = THANOS_ERR_CUDA;
+    cudaEvent_t* copied = evs;        // [2]
+    cudaEvent_t* consumed = evs + 2;  // [2]
+    cudaEvent_t start = evs[4];
+    if (st == THANOS_OK && (cudaEventRecord(start, stream) != cudaSuccess ||
+                            cudaStreamWaitEvent(copy_stream, start, 0) != cudaSuccess))
+      st = THANOS_ERR_CUDA;
     int64_t k = 0;
     for (int64_t t0 = 0; t0 < a && st == THANOS_OK; t0 += HOST_TOKEN_CHUNK, ++k) {
       int64_t nt = a - t0 < HOST_TOKEN_CHUNK ? a - t0 : HOST_TOKEN_CHUNK;
       int slot = (int)(k & 1);
       char* stage = base + L.Xstage + (size_t)slot * HOST_TOKEN_CHUNK * b * es;
-      if (k >= 2) cudaStreamWaitEvent(copy_stream, consumed[slot], 0);
-      if (cudaMemcpyAsync(stage, static_cast<const char*>(X_host) + (size_t)t0 * b * es,
-                          (size_t)nt * b * es, cudaMemcpyHostToDevice, copy_stream) != cudaSuccess)
+      bool ok = true;
+      if (k >= 2) ok = cudaStreamWaitEvent(copy_stream, consumed[slot], 0) == cudaSuccess;
+      ok = ok && cudaMemcpyAsync(stage, static_cast<const char*>(X_host) + (size_t)t0 * b * es,
+                                 (size_t)nt * b * es, cudaMemcpyHostToDevice,
+                                 copy_stream) == cudaSuccess;
+      ok = ok && cudaEventRecord(copied[slot], copy_stream) == cudaSuccess;
+      ok = ok && cudaStreamWaitEvent(stream, copied[slot], 0) == cudaSuccess;
+      if (!ok) {
         st = THANOS_ERR_CUDA;
-      cudaEventRecord(copied[slot], copy_stream);
-      cudaStreamWaitEvent(stream, copied[slot], 0);
-      if (st == THANOS_OK)
-        st = thanos_hessian_accumulate(H, b, stage, dtype, nt, b, ws, L.ws_bytes, stream);
-      cudaEventRecord(consumed[slot], stream);
+        break;
+      }
+      st = thanos_hessian_accumulate(H, b, stage, dtype, nt, b, ws, L.ws_bytes, stream);
+      if (st == THANOS_OK) {
+        // the accumulation's own status word (first word of its workspace) is cleared by the next
+        // chunk and overwritten by the later calls: keep the first failure in status[2]
+        fold_word_kernel<<<1, 1, 0, stream>>>(status + 2, static_cast<const int32_t*>(ws));
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) st = THANOS_ERR_CUDA;
+      }
+      if (cudaEventRecord(consumed[slot], stream) != cudaSuccess && st == THANOS_OK)
+        st = THANOS_ERR_CUDA;
     }
-    cudaStreamSynchronize(copy_stream);
-    cudaStreamDestroy(copy_stream);
-    for (int i = 0; i < 2; ++i) {
-      cudaEventDestroy(copied[i]);
-      cudaEventDestroy(consumed[i]);
+    // the staging buffers and the temporary stream / events are released only when every copy
+    // issued above has finished
+    if (copy_stream) {
+      cudaStreamSynchronize(copy_stream);
+      cudaStreamDestroy(copy_stream);
     }
-    cudaEventDestroy(start);
+    for (int i = 0; i < 5; ++i)
+      if (evs[i]) cudaEventDestroy(evs[i]);
     THANOS_TRY(st);
     THANOS_TRY(thanos_prepare_inverse(H, b, damp_rel, U, xnorm, ws, L.ws_bytes, status, stream));
   }
@@ -289,7 +322,11 @@ thanos_status_t thanos_prune_layer_host(const void* W_in_host, const void* X_hos
   int32_t st_host[4] = {0, 0, 0, 0};
   THANOS_CUDA(cudaMemcpyAsync(st_host, status, 16, cudaMemcpyDeviceToHost, stream));
   THANOS_CUDA(cudaStreamSynchronize(stream));
-  if (st_host[0] != 0 && stats_host->status == 0) {
+  if (st_host[2] != 0 && stats_host->status == 0) {  // Hessian accumulation (bounded wait ran out)
+    stats_host->status = st_host[2];
+    stats_host->err_index = -1;
+  }
+  if (st_host[0] != 0 && stats_host->status == 0) {  // factorisation
     stats_host->status = st_host[0];
     stats_host->err_index = st_host[1];
   }

@@ -343,8 +343,11 @@ hessian_tc2_kernel(const __grid_constant__ CUtensorMap tmap, const Params2 p) {
 
 // Clusters of two that can be resident at once (the grid is sized to it, persistent pairs).
 int max_active_pairs() {
-  static int cached = -1;
-  if (cached >= 0) return cached;
+  static std::atomic<int> cached_by_dev[64];  // 0 = not asked yet, else pairs + 1
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int have = cached_by_dev[dev].load(std::memory_order_relaxed);
+  if (have > 0) return have - 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * sm_count(), 1, 1);
   cfg.blockDim = dim3(NTHREADS, 1, 1);
@@ -361,7 +364,7 @@ int max_active_pairs() {
     cudaGetLastError();
     n = 0;
   }
-  cached = n;
+  cached_by_dev[dev].store(n + 1, std::memory_order_relaxed);
   return n;
 }
 

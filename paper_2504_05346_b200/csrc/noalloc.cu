@@ -1,16 +1,20 @@
 // thanos_prune_layer_noalloc: the block sweep for callers that cannot hand over a workspace.
 //
-// The sweep's scratch (inverse rows P, multipliers Lambda, histogram, sweep state, tie
-// prefixes, and the fp32 working copy for 16-bit weights) lives in one fixed array in the
-// library's device image instead of a caller buffer.  Everything else is the ordinary sweep.
+// The sweep's scratch (per-block matrices, the bf16 planes of the update operands, histogram,
+// sweep state, tie prefixes, row lists, the keys copied out of the selection window, and the fp32
+// working copy for 16-bit weights) lives in one fixed array in the library's device image instead
+// of a caller buffer.  Everything else is the ordinary sweep.
 #include <mutex>
 
 #include "common.cuh"
 
 namespace thanos {
 size_t prune_workspace_bytes(int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
-thanos_status_t validate_sweep_args(int64_t c, int64_t b, thanos_mode_t mode, double p, int32_t n,
-                                    int32_t m, int32_t B);
+thanos_status_t check_prune_layer_args(const void* W_in, const void* W_out, const uint8_t* mask_out,
+                                       thanos_dtype_t wdtype, int64_t c, int64_t b,
+                                       const float* factor, const float* xnorm, thanos_mode_t mode,
+                                       double p, int32_t n, int32_t m, int32_t B,
+                                       const thanos_stats_t* stats_dev);
 thanos_status_t prune_layer_impl(const void* W_in, void* W_out, uint8_t* mask_out,
                                  thanos_dtype_t wdtype, int64_t c, int64_t b, const float* U,
                                  const float* xnorm, thanos_mode_t mode, double p, int32_t n,
@@ -51,15 +55,22 @@ extern "C" thanos_status_t thanos_prune_layer_noalloc(
     const float* factor, const float* xnorm, thanos_mode_t mode, double p, int32_t n, int32_t m,
     int32_t B, thanos_stats_t* stats_dev, void* stream) {
   using namespace thanos;
-  if (!W_in || !W_out || !mask_out || !factor || !xnorm || !stats_dev)
-    return THANOS_ERR_INVALID_ARG;
-  if (wdtype != THANOS_F32 && wdtype != THANOS_BF16) return THANOS_ERR_DTYPE;
-  THANOS_TRY(validate_sweep_args(c, b, mode, p, n, m, B));
-  if (!aligned16(W_in) || !aligned16(W_out) || !aligned16(mask_out) || !aligned16(factor) ||
-      !aligned16(xnorm) || !aligned16(stats_dev))
-    return THANOS_ERR_ALIGNMENT;
+  THANOS_TRY(check_prune_layer_args(W_in, W_out, mask_out, wdtype, c, b, factor, xnorm, mode, p, n,
+                                    m, B, stats_dev));
   // the layer's scratch must fit the fixed array
   if (prune_workspace_bytes(c, b, B, wdtype) > kNoAllocScratchBytes) return THANOS_ERR_WORKSPACE;
+  // The scratch belongs to the CURRENT device; weights that live on another device would be
+  // swept with the wrong GPU's array (and launched on the wrong GPU).
+  {
+    int dev = -1;
+    cudaPointerAttributes attr;
+    if (cudaGetDevice(&dev) != cudaSuccess) return THANOS_ERR_CUDA;
+    if (cudaPointerGetAttributes(&attr, W_in) != cudaSuccess) {
+      cudaGetLastError();
+      return THANOS_ERR_INVALID_ARG;
+    }
+    if (attr.type == cudaMemoryTypeDevice && attr.device != dev) return THANOS_ERR_INVALID_ARG;
+  }
   void* scratch = nullptr;
   THANOS_TRY(scratch_for_current_device(&scratch));
   // The sweep itself resets what has to start at zero (histogram, sweep state) and writes every

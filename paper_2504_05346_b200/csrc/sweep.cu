@@ -485,6 +485,7 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       if (lane == 0) {
         st->lo = vs->lo + ((unsigned)bin << ((vs->wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2) - WINDOW_BINS_LOG2));
         st->k_rem = k - bel - before;
+        if (vs->cand_overflow) stats->select_rescans += 1;
       }
       next = PH_REFINE;
     } else {
@@ -712,6 +713,24 @@ __global__ void to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __re
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+// A single block step that continues a sweep: `stats` still holds what the previous block step
+// left (threshold of that block, whether a bracket has missed so far), so the selection starts
+// from the same bracket the whole-layer sweep would use.  A zeroed `stats` leaves the state on the
+// four radix passes.
+__global__ void seed_select_kernel(SweepState* st, const thanos_stats_t* stats) {
+  if (stats->n_blocks <= 0) return;
+  const int wide = stats->select_misses > 0 ? 1 : 0;
+  const unsigned tau = stats->last_threshold_bits;
+  const unsigned half_window = 1u << ((wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2) - 1);
+  st->wide = wide;
+  if (tau >= half_window) {
+    st->tau_prev = tau;
+    st->have_prev = 1;
+    st->lo = tau - half_window;
+    st->phase = PH_BRACKET;
+  }
 }
 
 __global__ void init_sweep_kernel(SweepState* st, thanos_stats_t* stats, long long r) {
@@ -1006,6 +1025,10 @@ thanos_status_t prune_block_impl(float* Wc, uint8_t* mask, int64_t c, int64_t b,
   THANOS_CUDA(cudaMemsetAsync(w.hist, 0, HIST_BINS * sizeof(unsigned), stream));
   THANOS_CUDA(cudaMemsetAsync(w.st, 0, sizeof(SweepState), stream));
   THANOS_CUDA(cudaMemsetAsync(w.tc_status, 0, 16, stream));
+  if (mode == THANOS_UNSTRUCTURED) {
+    seed_select_kernel<<<1, 1, 0, stream>>>(w.st, stats);
+    THANOS_CHECK_LAUNCH();
+  }
   THANOS_TRY(prepare_blocks(U, (int)b, B, w, stream));
   THANOS_TRY(block_step(Wc, mask, (int)c, (int)b, xnorm, mode, n, m, B, (int)j1, r_dev, w, stats,
                         stream));

@@ -118,13 +118,16 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// SM count of the current device (cached per device).
 inline int sm_count() {
-  static int n = 0;
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NUM_SMS;
+  int n = cached[dev].load(std::memory_order_relaxed);
   if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = NUM_SMS;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = NUM_SMS;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
   return n;
 }

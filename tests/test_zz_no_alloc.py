@@ -55,6 +55,36 @@ def test_noalloc_matches_prune_layer_on_consecutive_calls(T):
     assert a1[2].n_pruned == 64 * 256 // 2 and a2[2].n_pruned == 48 * 128 // 2
 
 
+def test_noalloc_calls_leave_device_memory_untouched(T):
+    """With the outputs and the statistics buffer created beforehand, a call must not change the
+    amount of device memory in use: neither PyTorch's allocator nor the driver's free-memory count
+    moves across three calls (after a first call that looks up the scratch address), and calls
+    share no state beyond the scratch (identical statistics for identical inputs)."""
+    U, xn = _factor(T, 256, seed=6)
+    W = WL.make_weight(64, 256, "f32", seed=74).to(DEV)
+    out = torch.empty_like(W)
+    mask = torch.empty(W.shape, dtype=torch.uint8, device=DEV)
+    stats = [torch.zeros(64, dtype=torch.uint8, device=DEV) for _ in range(3)]
+    lib = T.load_library()
+    args = lambda st: (W.data_ptr(), out.data_ptr(), mask.data_ptr(), T.F32, 64, 256, U.data_ptr(),
+                       xn.data_ptr(), T.UNSTRUCTURED, 0.5, 0, 0, 64, st.data_ptr(),
+                       torch.cuda.current_stream().cuda_stream)
+    warm = torch.zeros(64, dtype=torch.uint8, device=DEV)
+    assert lib.thanos_prune_layer_noalloc(*args(warm)) == 0      # first call: address look-up
+    torch.cuda.synchronize()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    free0, _ = torch.cuda.mem_get_info()
+    for st in stats:
+        assert lib.thanos_prune_layer_noalloc(*args(st)) == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert free1 == free0
+    assert torch.equal(stats[0], stats[1]) and torch.equal(stats[1], stats[2])
+    ref = T.prune_layer(W, U, xn, T.UNSTRUCTURED, p=0.5, B=64)
+    assert torch.equal(mask, ref[1]) and torch.equal(out, ref[0])
+
+
 def test_noalloc_refuses_layers_beyond_its_fixed_scratch(T):
     U, xn = _factor(T, 256, seed=5)
     big = torch.zeros((8192, 256), dtype=torch.float32, device=DEV)  # needs > 4 MiB of scratch
