@@ -33,10 +33,11 @@ UNIT = "weights/s"
 TOKEN_CHUNK = 262144  # tokens per thanos_hessian_accumulate call (the activations are resident)
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the Hessian kernel from
-# the ncu captures summarised under profiles/ (hessian_tc2_kernel_*.md): width b -> (bytes, tokens
-# of the captured launch).  A launch streams X once per wave of tile pairs, so its traffic grows in
-# proportion to its tokens; the figure reported with the bench line is scaled that way.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the Hessian kernel,
+# taken once with ncu on launches short enough to capture: width b -> (bytes, tokens of the captured
+# launch).  A launch streams X once per wave of tile pairs, so its traffic grows in proportion to
+# its tokens; the figure reported with the bench line is scaled that way.  Set an entry to None
+# when the kernel has changed since its counters were taken (the line then reports null).
 HESSIAN_DRAM_CAPTURE = {4096: (2.083e9, 65536), 11008: (4.567e9, 16384)}
 
 
@@ -45,7 +46,7 @@ def hessian_traffic_per_launch(launch_shapes):
     captured."""
     tot = 0.0
     for b, tok in launch_shapes:
-        if b not in HESSIAN_DRAM_CAPTURE:
+        if HESSIAN_DRAM_CAPTURE.get(b) is None:
             return None
         byt, cap_tok = HESSIAN_DRAM_CAPTURE[b]
         tot += byt * tok / cap_tok
@@ -177,6 +178,139 @@ def mode_args(cfg, T):
     return dict(mode=T.NM, n=cfg.n, m=cfg.m)
 
 
+def select_mode(cfg, index: int):
+    """index 0: the configuration's own sparsity mode; k > 0: its k-th additional mode (the
+    LLaMA-2-70B-shaped set is also pruned to 60 % unstructured)."""
+    if index == 0:
+        return cfg
+    kind, val = cfg.extra_modes[index - 1]
+    if kind == "unstructured":
+        return dataclasses.replace(cfg, mode="unstructured", p=float(val))
+    n, m = val
+    return dataclasses.replace(cfg, mode="nm", n=int(n), m=int(m))
+
+
+def kernel_trace(fn):
+    """Runs fn() under a CUPTI activity trace (torch.profiler, device activities only) and returns
+    {kernel name: [launches, device ms]} plus the copies / memsets; None when no trace can be had.
+    Used for ONE extra, untimed step whose calls are issued on a single stream, so that the step's
+    time can be split by kernel; nothing measured under the trace is reported as a bench value."""
+    try:
+        from torch.profiler import ProfilerActivity, profile
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            fn()
+            torch.cuda.synchronize()
+        agg = {}
+        for e in prof.events():
+            if e.device_type == torch.autograd.DeviceType.CUDA:
+                d = agg.setdefault(e.name, [0, 0.0])
+                d[0] += 1
+                d[1] += e.device_time * 1e-3
+        return agg or None
+    except Exception:
+        return None
+
+
+def short_kernel_name(name: str) -> str:
+    n = name.replace("thanos::(anonymous namespace)::", "").replace("void ", "")
+    return n.split("(")[0]
+
+
+def measure_fp32_peak(T, dev):
+    """Plain fp32 FMA throughput of this device from the library's FMA-chain kernel (best of 5
+    launches of about a millisecond, CUDA events): the roofline of the per-row solves."""
+    ctas = 148 * 8
+    out = torch.empty(ctas * 256, dtype=torch.float32, device=dev)
+    T.fp32_fma_probe(out, ctas, 64)
+    torch.cuda.synchronize()
+    best = 0.0
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        flop = T.fp32_fma_probe(out, ctas, 16384)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, flop / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best
+
+
+def solve_flop(masks, cfg):
+    """Arithmetic of the per-row systems of one step from the masks it produced: per row and
+    block, with s removed of B and n = min(s, B - s) unknowns (direct or complement form),
+    n^3 / 3 + 2 n^2 + 2 s (B - s) floating-point operations (factorisation, two triangular
+    solves, the product that spreads the solution over the block)."""
+    tot = 0.0
+    B = cfg.B
+    for M in masks:
+        c, b = M.shape
+        nb = b // B
+        if nb == 0:
+            continue
+        s_ = M[:, : nb * B].reshape(c, nb, B).sum(dim=2, dtype=torch.int32).double()
+        n_ = torch.minimum(s_, B - s_)
+        tot += float((n_ ** 3 / 3.0 + 2.0 * n_ ** 2 + 2.0 * s_ * (B - s_)).sum())
+    return tot
+
+
+def roofline_by_kernel(trace_factor, trace_sweep, cfg, peaks, fp32_peak, masks, n_inputs_by_b):
+    """Fractions of the governing roofline for the kernels next to the Hessian, from the per-kernel
+    device times of one serialised step (trace_factor: Hessians + factorisations, trace_sweep: the
+    sweeps) and the algorithmic work of that step."""
+    def t_of(trace, key):
+        if not trace:
+            return None, 0
+        ms = sum(v[1] for k, v in trace.items() if key in k)
+        n = sum(v[0] for k, v in trace.items() if key in k)
+        return (ms if n else None), n
+
+    out = {}
+    unstructured = cfg.mode == "unstructured"
+    B = cfg.B
+    resid_elems = 0.0   # sum over layers and blocks of c (b - j1): one look at the residual per block
+    upd_elems = 0.0     # sum over layers and blocks of c (b - j2): what a block's update changes
+    for L in cfg.layers:
+        for j1 in range(0, L.b, B):
+            j2 = min(L.b, j1 + B)
+            resid_elems += float(L.c) * (L.b - j1)
+            upd_elems += float(L.c) * (L.b - j2)
+    hbm = peaks["hbm_gbs"]
+    if unstructured:
+        ms, n = t_of(trace_sweep, "select_pass_kernel")
+        if ms:
+            ach = 4.0 * resid_elems / (ms * 1e-3) / 1e9
+            out["select_pass_kernel"] = {
+                "bound": "hbm", "achieved": round(ach, 1), "peak": hbm, "unit": "GB/s",
+                "frac": round(ach / hbm, 4), "ms_per_step": round(ms, 3), "launches": n,
+                "work": "4 c (b - j1) bytes per block: one read of the residual"}
+    ms, n = t_of(trace_sweep, "tc_gemm_kernel")
+    if ms:
+        ach = 8.0 * upd_elems / (ms * 1e-3) / 1e9
+        out["tc_gemm_kernel (sweep update)"] = {
+            "bound": "hbm", "achieved": round(ach, 1), "peak": hbm, "unit": "GB/s",
+            "frac": round(ach / hbm, 4), "ms_per_step": round(ms, 3), "launches": n,
+            "work": "8 c (b - j2) bytes per block: the residual read and written once"}
+    ms, n = t_of(trace_factor, "tc_gemm_kernel")
+    if ms:
+        flop = sum(k * (2.0 / 3.0) * float(b) ** 3 for b, k in n_inputs_by_b.items())
+        ach = flop / (ms * 1e-3) / 1e12
+        pk = peaks["bf16_tflops_sustained"]
+        out["tc_gemm_kernel (factorisation)"] = {
+            "bound": "tensor", "achieved": round(ach, 2), "peak": pk, "unit": "TFLOP/s",
+            "frac": round(ach / pk, 4), "ms_per_step": round(ms, 3), "launches": n,
+            "work": "2/3 b^3 useful FLOP per factorisation (Cholesky + triangular inverse); the "
+                    "kernel executes six bf16-plane products per fp32 product"}
+    ms, n = t_of(trace_sweep, "solve_rows")
+    if ms and fp32_peak:
+        ach = solve_flop(masks, cfg) / (ms * 1e-3) / 1e12
+        out["solve_rows kernels"] = {
+            "bound": "alu", "achieved": round(ach, 2), "peak": round(fp32_peak, 2),
+            "unit": "TFLOP/s", "frac": round(ach / fp32_peak, 4), "ms_per_step": round(ms, 3),
+            "launches": n, "peak_source": "measured: FMA-chain kernel of this library, this run",
+            "work": "n^3/3 + 2 n^2 + 2 s (B - s) FLOP per row and block, n = min(s, B - s), "
+                    "counted from the step's masks"}
+    return out
+
+
 # ------------------------------------------------------------------------------------------
 def run_ours(args):
     import torch.distributed as dist
@@ -197,7 +331,7 @@ def run_ours(args):
         dist.barrier()
     T.load_library()
 
-    cfg = WL.CONFIGS[args.workload]
+    cfg = select_mode(WL.CONFIGS[args.workload], args.mode_index)
     a = args.tokens or cfg.a
     dt = T.BF16 if cfg.dtype == "bf16" else T.F32
     margs = mode_args(cfg, T)
@@ -231,59 +365,59 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     hess_events = []  # (start, end, flops, (b, tokens)) per thanos_hessian_accumulate call
-    phase_events = {"hessian": [], "prepare": [], "prune": []}
+    hess_status = {iid: torch.zeros(1, dtype=torch.int32, device=dev) for iid in in_ids}
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    def one_step(record):
+    def one_step(record, serial=False, do_factor=True, do_sweep=True):
+        """One pass over the layer set.  `serial` issues every call on the main stream (used by
+        the untimed per-kernel trace); `do_factor` / `do_sweep` select the two halves of the step
+        (Hessians + factorisations, sweeps) for that trace."""
         stats_all = [None] * len(cfg.layers)
-        # the Hessians fill the whole GPU by themselves: one after the other on the main stream
-        for iid in in_ids:
-            X = inputs[iid]
-            b = X.shape[1]
-            H = Hbuf[iid]
-            e0 = ev()
-            e0.record(main)
-            H.zero_()
-            for t0 in range(0, a, TOKEN_CHUNK):
-                xc = X[t0:t0 + TOKEN_CHUNK]
-                if record:
-                    hs, he = ev(), ev()
-                    hs.record(main)
-                T.hessian_accumulate(H, xc, workspace=ws_in[iid])
-                if record:
-                    he.record(main)
-                    hess_events.append((hs, he, float(xc.shape[0]) * b * (b + 1),
-                                        (b, int(xc.shape[0]))))
-            e1 = ev()
-            e1.record(main)
-            if record:
-                phase_events["hessian"].append((e0, e1))
-        e_h = ev()
-        e_h.record(main)
-        # factorisations and sweeps: one stream per input, then one per layer
         ready = {}
-        for iid in in_ids:
-            s = s_in[iid]
-            s.wait_event(e_h)
-            with torch.cuda.stream(s):
-                e1 = ev()
-                e1.record(s)
-                T.prepare_inverse(Hbuf[iid], cfg.damp_rel, workspace=ws_in[iid], check=False,
-                                  factor=Ubuf[iid], xnorm=xnbuf[iid])
-                e2 = ev()
-                e2.record(s)
-                ready[iid] = e2
-            if record:
-                phase_events["prepare"].append((e1, e2))
+        if do_factor:
+            # the Hessians fill the whole GPU by themselves: one after the other on the main stream
+            for iid in in_ids:
+                X = inputs[iid]
+                b = X.shape[1]
+                H = Hbuf[iid]
+                H.zero_()
+                for t0 in range(0, a, TOKEN_CHUNK):
+                    xc = X[t0:t0 + TOKEN_CHUNK]
+                    if record:
+                        hs, he = ev(), ev()
+                        hs.record(main)
+                    T.hessian_accumulate(H, xc, workspace=ws_in[iid])
+                    if record:
+                        he.record(main)
+                        hess_events.append((hs, he, float(xc.shape[0]) * b * (b + 1),
+                                            (b, int(xc.shape[0]))))
+                    # the call's status word sits in the workspace the factorisation reuses
+                    torch.maximum(hess_status[iid], ws_in[iid][:4].view(torch.int32),
+                                  out=hess_status[iid])
+            e_h = ev()
+            e_h.record(main)
+            # factorisations: one stream per input
+            for iid in in_ids:
+                s = main if serial else s_in[iid]
+                s.wait_event(e_h)
+                with torch.cuda.stream(s):
+                    T.prepare_inverse(Hbuf[iid], cfg.damp_rel, workspace=ws_in[iid], check=False,
+                                      factor=Ubuf[iid], xnorm=xnbuf[iid])
+                    e2 = ev()
+                    e2.record(s)
+                    ready[iid] = e2
+        if not do_sweep:
+            for e in ready.values():
+                main.wait_event(e)
+            return stats_all
         done = []
         for i, L in enumerate(cfg.layers):
-            s = s_layer[i]
-            s.wait_event(ready[L.input_id])
+            s = main if serial else s_layer[i]
+            if L.input_id in ready:
+                s.wait_event(ready[L.input_id])
             with torch.cuda.stream(s):
-                p0 = ev()
-                p0.record(s)
                 _, _, st = T.prune_layer(weights[i], Ubuf[L.input_id], xnbuf[L.input_id], B=cfg.B,
                                          workspace=ws_layer[i], out=outs[i], mask=masks[i],
                                          read_stats=False, **margs)
@@ -291,8 +425,6 @@ def run_ours(args):
                 p1.record(s)
             stats_all[i] = st
             done.append(p1)
-            if record:
-                phase_events["prune"].append((p0, p1))
         for e in done:
             main.wait_event(e)
         return stats_all
@@ -322,10 +454,15 @@ def run_ours(args):
     ms_total = t_start.elapsed_time(t_end)
     ms_total = max_over_ranks(ms_total, dev)
     # device status of the last step
+    select_misses = 0
     for st in stats_last:
         ps = T.PruneStats.from_bytes(bytes(st.cpu().numpy().tobytes()))
         if ps.status != 0:
             raise RuntimeError("device status %d in prune_layer" % ps.status)
+        select_misses += ps.select_misses
+    for iid, hs in hess_status.items():
+        if int(hs.item()) != 0:
+            raise RuntimeError("device status %d in hessian_accumulate" % int(hs.item()))
 
     nweights = layer_set_weights(cfg)
     ms_per_step = ms_total / args.steps
@@ -338,13 +475,32 @@ def run_ours(args):
     traffic = hessian_traffic_per_launch([ev[3] for ev in hess_events])
     achieved = h_flops / (h_ms * 1e-3) / 1e12 if h_ms > 0 else 0.0
     peak = peaks["bf16_tflops_sustained"]
-    phase_ms = {k: sum(s.elapsed_time(e) for s, e in v) / args.steps for k, v in phase_events.items()}
     roofline = {"kernel": "hessian_tc2_kernel (thanos_hessian_accumulate)", "bound": "tensor", "achieved": round(achieved, 2),
                 "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
                 "peak_source": peaks["source"] + " (sustained bf16)",
                 "traffic": None if traffic is None else round(traffic),
                 "traffic_unit": "DRAM bytes per launch, ncu capture of a shorter launch scaled by tokens",
                 "launches": len(hess_events), "avg_launch_ms": round(h_ms / max(1, len(hess_events)), 4)}
+
+    # ---- the rest of the step by kernel: ONE extra untimed step, every call on one stream, under
+    #      a device-activity trace, in two halves so that the tensor-core products of the
+    #      factorisations and of the sweeps are told apart
+    by_kernel, kernel_ms, fp32_peak = None, None, None
+    if rank == 0 and not args.no_kernel_split:
+        fp32_peak = measure_fp32_peak(T, dev)
+        tr_f = kernel_trace(lambda: one_step(False, serial=True, do_sweep=False))
+        tr_s = kernel_trace(lambda: one_step(False, serial=True, do_factor=False))
+        if tr_f and tr_s:
+            n_by_b = {}
+            for iid in in_ids:
+                n_by_b[inputs[iid].shape[1]] = n_by_b.get(inputs[iid].shape[1], 0) + 1
+            by_kernel = roofline_by_kernel(tr_f, tr_s, cfg, peaks, fp32_peak, masks, n_by_b)
+            kernel_ms = {}
+            for half, tr in (("hessians+factorisations", tr_f), ("sweeps", tr_s)):
+                kernel_ms[half] = {short_kernel_name(k): [v[0], round(v[1], 3)]
+                                   for k, v in sorted(tr.items(), key=lambda kv: -kv[1][1])
+                                   if v[1] >= 0.05}
+                kernel_ms[half]["total_ms"] = round(sum(v[1] for v in tr.values()), 3)
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -368,13 +524,19 @@ def run_ours(args):
                                       cfg.B, cfg.damp_rel),
                        "weights_per_step": nweights, "l2": "inputs larger than L2",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "streams": ("one per layer input and one per layer (calls overlap; "
-                                   "phase_ms_per_step sums per-call times)") if overlap else "one",
+                       "streams": "one per layer input and one per layer (calls overlap)"
+                       if overlap else "one",
                        "token_chunk": TOKEN_CHUNK},
             "ms_per_layer": ms_per_step / len(cfg.layers),
-            "phase_ms_per_step": {k: round(v, 3) for k, v in phase_ms.items()},
+            "select_misses_last_step": int(select_misses),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "roofline_by_kernel": by_kernel,
+            "fp32_fma_peak_tflops_measured": None if fp32_peak is None else round(fp32_peak, 2),
+            "kernel_ms_serialised_step": kernel_ms,
+            "kernel_ms_note": "device time per kernel [launches, ms] of one extra untimed step "
+                              "issued on a single stream, from a device-activity trace; the timed "
+                              "steps overlap these calls on several streams",
+            "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
     if world > 1:
@@ -516,7 +678,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg = WL.CONFIGS[args.workload]
+    cfg = select_mode(WL.CONFIGS[args.workload], args.mode_index)
     vals, last = [], None
     t0 = time.perf_counter()
     for i in range(args.warmup + args.steps):
@@ -543,8 +705,8 @@ def run_reference(args):
 
 
 def run_single_layer(args):
-    """One layer (c, b) with `a` calibration tokens through the three calls, `--reps` times; the
-    small, fixed command the ncu captures under profiles/ were taken with."""
+    """One layer (c, b) with `a` calibration tokens through the three calls, `--reps` times: a
+    small, fixed workload for profiler captures of single kernels."""
     import paper_2504_05346_b200 as T
     from paper_2504_05346_b200 import build as B_
 
@@ -593,6 +755,20 @@ def run_single_layer(args):
     print(json.dumps({"single_layer": [c, b, a], "workload": cfg.name, "runs": out}))
 
 
+def replica_launch_command(n_gpus: int, argv, port: int):
+    """Command that starts `n_gpus` replicas of this script, one process per GPU, on this node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+            "--nproc-per-node", str(n_gpus), "--master-addr", "127.0.0.1",
+            "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def _free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return int(sk.getsockname()[1])
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -608,6 +784,11 @@ def main():
     ap.add_argument("--e2e-workers", type=int, default=3,
                     help="host threads (each with a stream and an arena) of the end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-split", action="store_true",
+                    help="skip the extra untimed step that splits the step's time by kernel")
+    ap.add_argument("--mode-index", type=int, default=0,
+                    help="0: the workload's own sparsity mode; k: its k-th additional mode "
+                         "(llama2_70b: 1 = 60 %% unstructured)")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
     ap.add_argument("--single-layer", default="", metavar="C,B,A",
                     help="profile driver: one c x b layer with a tokens instead of the layer set")
@@ -623,6 +804,13 @@ def main():
     if args.single_layer:
         run_single_layer(args)
         return
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1:
+        # not under a launcher: start one replica per GPU and hand over
+        cmd = replica_launch_command(args.gpus, sys.argv[1:], _free_port())
+        sys.exit(subprocess.call(cmd))
+    if world_env is not None and int(world_env) != args.gpus:
+        sys.exit("bench.py: --gpus %d but the launcher started %s ranks" % (args.gpus, world_env))
     if args.impl == "reference":
         run_reference(args)
     else:

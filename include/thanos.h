@@ -307,6 +307,16 @@ thanos_status_t thanos_dense_product(float* D, int64_t ldd, const float* A, int6
                                      void* workspace, size_t ws_bytes, void* stream);
 size_t thanos_dense_product_workspace(int64_t M, int64_t N, int64_t K);
 
+/*
+ * Measurement aid (the paper has no counterpart): launches `ctas` CTAs of 256 threads that each
+ * run 16 independent chains of 4 * iters dependent fp32 FMAs and store one float per thread to
+ * `out` (device, at least ctas * 256 floats).  *flop_out (host, may be NULL) receives the
+ * floating-point operations of the launch, 2 per FMA.  Timed by the caller with events, this
+ * gives the plain fp32 arithmetic peak of the device -- the roofline of the per-row solves.
+ */
+thanos_status_t thanos_fp32_fma_probe(float* out, int64_t out_elems, int32_t ctas, int32_t iters,
+                                      double* flop_out, void* stream);
+
 /* Minimum workspace in bytes for a call (see thanos_ws_which_t); 0 for unsupported shapes. */
 size_t thanos_workspace_bytes(int32_t which, int64_t c, int64_t b, int32_t B, thanos_dtype_t dtype);
 

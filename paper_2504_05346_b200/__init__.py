@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     prune_layer_host,
     prune_layer_noalloc,
     dense_product,
+    fp32_fma_probe,
     prune_layer_outliers,
     prune_layer_structured,
     workspace_bytes,

@@ -111,6 +111,8 @@ def load_library():
     lib.thanos_dense_product.restype = i32
     lib.thanos_dense_product_workspace.argtypes = [i64, i64, i64]
     lib.thanos_dense_product_workspace.restype = sz
+    lib.thanos_fp32_fma_probe.argtypes = [vp, i64, i32, i32, ctypes.POINTER(ctypes.c_double), vp]
+    lib.thanos_fp32_fma_probe.restype = i32
     lib.thanos_workspace_bytes.argtypes = [i32, i64, i64, i32, i32]
     lib.thanos_workspace_bytes.restype = sz
     lib.thanos_status_string.argtypes = [i32]
@@ -351,6 +353,19 @@ def prune_layer_noalloc(W: torch.Tensor, factor: torch.Tensor, xnorm: torch.Tens
     if st.status != 0:
         raise ThanosError(st.status, "thanos_prune_layer_noalloc (row %d)" % st.err_index)
     return out, mask, st
+
+
+def fp32_fma_probe(out: torch.Tensor, ctas: int, iters: int, stream=None) -> float:
+    """thanos_fp32_fma_probe: enqueues the FMA-chain kernel; returns its floating-point
+    operation count (time it with CUDA events around this call)."""
+    lib = load_library()
+    _check_dev(out)
+    flop = ctypes.c_double(0.0)
+    with _on(out):
+        _check(lib.thanos_fp32_fma_probe(out.data_ptr(), out.numel(), ctas, iters,
+                                         ctypes.byref(flop), _stream_ptr(stream)),
+               "thanos_fp32_fma_probe")
+    return float(flop.value)
 
 
 def dense_product(A: torch.Tensor, B: torch.Tensor, b_transposed: bool = False, alpha: float = 1.0,

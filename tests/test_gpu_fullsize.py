@@ -223,14 +223,15 @@ def test_hessian_one_call_of_the_benchmark_length(T):
 
 
 # ------------------------------------------------------------------------------ wide layers
-def _rows_times_matrix(rows64, M32, add_diag=0.0, chunk=2048):
+def _rows_times_matrix(rows64, M32, add_diag=0.0, chunk=2048, absolute=False):
     """rows64 [k, n] (float64) times the fp32 matrix M32 [n, n] (a host tensor) + add_diag * rows64,
-    in float64, converting M32 a column strip at a time."""
+    in float64, converting M32 a column strip at a time (`absolute`: of the absolute values)."""
     n = M32.shape[0]
     out = np.empty((rows64.shape[0], n))
     for c0 in range(0, n, chunk):
         c1 = min(n, c0 + chunk)
-        out[:, c0:c1] = rows64 @ M32[:, c0:c1].double().numpy()
+        strip = M32[:, c0:c1].double().numpy()
+        out[:, c0:c1] = rows64 @ (np.abs(strip) if absolute else strip)
     return out + add_diag * rows64
 
 
@@ -265,13 +266,21 @@ def _kkt_first_block(T, W, U, xn, H32, lam, mode, n, m, B, r0, rows):
     Mq = mask[rows].cpu().numpy().astype(bool)
     assert not Mq[:, B:].any()
     g = _rows_times_matrix(delta, H32, add_diag=lam)
+    # g_j is a sum with heavy cancellation (columns of high-energy features carry terms 1e3 times
+    # the result): its natural scale is sum_i |delta_i| |H_d[i, j]|
+    scale = _rows_times_matrix(np.abs(delta), H32, add_diag=lam, absolute=True)
+    worst = 0.0
     for k in range(len(rows)):
         q = Mq[k]
         if not q.any():
             assert not delta[k].any()
             continue
         assert np.array_equal(delta[k][q], -_np64(W[rows[k]])[q])
-        assert np.max(np.abs(g[k][~q])) <= 2e-3 * np.max(np.abs(g[k][q]))
+        worst = max(worst, float(np.max(np.abs(g[k][~q]) / scale[k][~q])))
+        # the check has teeth: on the removed positions the gradient is far from cancelling
+        assert np.max(np.abs(g[k][q]) / scale[k][q]) >= 1e-2
+    print("first block, b = %d: largest |delta H_d| / (|delta| |H_d|) on kept weights %.2e" % (b, worst))
+    assert worst <= 1e-4
     return mask
 
 
@@ -326,7 +335,7 @@ def test_llama3_8b_down_projection_width(T):
     lam = cfg.damp_rel * float(np.mean(np.diag(H32.numpy()).astype(np.float64)))
     err = _factor_identity_error(U32, H32, lam, [0, 5000, b - 1])
     print("max |U H_d U^T - I| on sampled rows, b = %d: %.2e" % (b, err))
-    assert err <= 2e-3
+    assert err <= 1e-4
     rows = [0, 100, c - 1]
     _late_block_literal(T, W, U, xn, H32, lam, (cfg.n, cfg.m), B, b - 2048, rows)
     _kkt_first_block(T, W, U, xn, H32, lam, T.NM, cfg.n, cfg.m, B, 0, rows)
@@ -352,7 +361,7 @@ def test_llama2_70b_down_projection_width(T, mode):
         U32 = U.cpu()
         err = _factor_identity_error(U32, H32, lam, [0, 9999, b - 1])
         print("max |U H_d U^T - I| on sampled rows, b = %d: %.2e" % (b, err))
-        assert err <= 2e-3
+        assert err <= 1e-4
         del U32
         _late_block_literal(T, W, U, xn, H32, lam, (2, 4), B, b - 2048, rows)
         _kkt_first_block(T, W, U, xn, H32, lam, T.NM, 2, 4, B, 0, rows)

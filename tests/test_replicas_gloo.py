@@ -57,3 +57,36 @@ def test_single_process_needs_no_group():
 
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.whole_job_rate(10, 2, 1, 4.0) == 10 * 2 / 4e-3
+
+
+def test_gpus_flag_builds_a_launch_of_that_many_replicas(monkeypatch):
+    """`bench.py --gpus 2` outside a launcher starts two ranks of itself on this node (it used to
+    run one replica whatever the flag said); under a launcher a rank count that disagrees with
+    the flag is an error."""
+    sys.path.insert(0, ROOT)
+    import bench
+
+    cmd = bench.replica_launch_command(2, ["--gpus", "2", "--steps", "4"], 29511)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "2"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "29511"
+    assert cmd[-4:] == ["--gpus", "2", "--steps", "4"] and cmd[-5].endswith("bench.py")
+
+    calls = []
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(bench.subprocess, "call", lambda c: calls.append(c) or 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "1"])
+    try:
+        bench.main()
+    except SystemExit as e:
+        assert e.code == 0
+    assert len(calls) == 1 and calls[0][calls[0].index("--nproc-per-node") + 1] == "2"
+
+    monkeypatch.setenv("WORLD_SIZE", "4")
+    try:
+        bench.main()
+        raised = False
+    except SystemExit as e:
+        raised = e.code not in (0, None)
+    assert raised
