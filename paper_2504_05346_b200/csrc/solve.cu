@@ -461,6 +461,12 @@ thanos_status_t launch_fast(float* Wc, const uint8_t* mask, const float* G, cons
 
 }  // namespace
 
+int tile_solve_max_unknowns();
+thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                  int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b,
+                                  int j1, int Bw, int ldd, int n_max, const int* row_lists,
+                                  const unsigned* list_counts, int fixed_kind, int report_max_s,
+                                  thanos_stats_t* stats, cudaStream_t stream);
 int cta_solve_max_unknowns();
 thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
                                  int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b, int j1,
@@ -468,8 +474,9 @@ thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G,
                                  const unsigned* list_counts, int fixed_kind, int report_max_s,
                                  thanos_stats_t* stats, cudaStream_t stream);
 
-// Systems of up to 159 unknowns go to the warp-per-row kernel, larger ones to the CTA-per-row
-// kernel; n_small_max is the largest min(|q|, |k|) a row can have.
+// Systems of up to 64 unknowns go to the warp-per-row tile kernel (solve_tile.cu), up to 159 to the
+// warp-per-row panel kernel above, larger ones to the CTA-per-row kernel; n_small_max is the
+// largest min(|q|, |k|) a row can have.
 bool solve_supported(int s_direct_max, int n_small_max) {
   (void)s_direct_max;
   return n_small_max <= cta_solve_max_unknowns();
@@ -495,6 +502,10 @@ thanos_status_t launch_block_solve(float* Wc, const uint8_t* mask, const float* 
   if (n_small + 1 > 160 || (n_small + 1 > 96 && Bw <= 256))
     return launch_cta_solve(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                             fixed_kind, rep, stats, stream);
+  // up to 64 unknowns: the warp-per-row tile kernel with tensor-core trailing updates
+  if (n_small <= tile_solve_max_unknowns() && Bw <= 1024)
+    return launch_tile_solve(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
+                             fixed_kind, rep, stats, stream);
   if (n_small + 1 <= 32)
     return launch_fast<1>(Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, n_small, rl, lc,
                           fixed_kind, rep, stats, stream);

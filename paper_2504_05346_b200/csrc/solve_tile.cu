@@ -1,0 +1,638 @@
+// Per-row constrained solve of one block step (Eqs. 5-8) for systems of up to 64 unknowns: one warp
+// per row, tile Cholesky whose panel and trailing products run on the tensor cores.
+//
+// Same mathematics as solve.cu (direct form on G for rows with |q| <= |k|, complement form on S
+// otherwise).  The gathered matrix lives in shared memory as the lower triangle of 16 x 16 fp32
+// tiles (tile_ops.cuh).  Per tile column K the warp
+//   factors the diagonal tile with warp shuffles -- lanes 0..15 hold its rows, lanes 16..31 the
+//   rows of the identity, and the same column operations leave L_KK in the former and L_KK^{-T}
+//   in the latter (kept in the unused upper triangle of the tile);
+//   forms the panel below it as a product, L_IK = A_IK L_KK^{-T};
+//   and subtracts L_IK L_JK^T from every trailing tile.
+// The products use mma.sync m16n8k16: fp32 tiles are split into three bf16 planes in registers
+// (24 significant bits), six plane products are accumulated in fp32; the accumulator layout of a
+// panel product is the A-operand layout of the trailing product, so a panel tile goes from one to
+// the other without leaving the registers.  The right-hand side is a vector of its own; with the
+// inverses of the diagonal tiles both substitutions are 16 x 16 matrix-vector products per tile
+// row, and the only serial chains left are the four diagonal factorisations.
+#include "common.cuh"
+#include "tile_ops.cuh"
+
+namespace thanos {
+
+namespace {
+
+using tile::chunk_off;
+using tile::elem_off;
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int TILE_T_MAX = 4;  // tile rows: systems of up to 64 unknowns
+
+__device__ __forceinline__ int tbase(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
+
+struct TileSolveLayout {
+  int mat_floats;      // shared copy of G or S (0 when it stays in global memory)
+  int ldm;
+  int tiles_floats;
+  int per_warp_bytes;
+};
+
+__host__ __device__ inline TileSolveLayout tile_solve_layout(int Bw, int T, bool mat_in_smem) {
+  TileSolveLayout L;
+  L.ldm = mat_in_smem ? (Bw | 1) : 0;
+  L.mat_floats = mat_in_smem ? ((Bw * L.ldm + 3) & ~3) : 0;
+  L.tiles_floats = (T * (T + 1) / 2) * 256;
+  // tiles, invd[16 T], yv[16 T + 16], wblk[Bw], dvec[Bw], two index lists of Bw + 16 shorts
+  const int bytes = 4 * (L.tiles_floats + 16 * T + 16 * T + 16 + 2 * Bw) + 2 * 2 * (Bw + 16);
+  L.per_warp_bytes = (bytes + 15) & ~15;
+  return L;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+  // no side effects beyond its outputs: not volatile, so that independent chains interleave
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// (x0, x1) -> three words of two bf16 each (x0 in the low half): x = p0 + p1 + p2 to 24 bits
+__device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& p0, uint32_t& p1,
+                                           uint32_t& p2) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  p0 = *reinterpret_cast<const uint32_t*>(&h);
+  x0 -= __uint_as_float(p0 << 16);
+  x1 -= __uint_as_float(p0 & 0xffff0000u);
+  h = __floats2bfloat162_rn(x0, x1);
+  p1 = *reinterpret_cast<const uint32_t*>(&h);
+  x0 -= __uint_as_float(p1 << 16);
+  x1 -= __uint_as_float(p1 & 0xffff0000u);
+  h = __floats2bfloat162_rn(x0, x1);
+  p2 = *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Fragment of a 16 x 16 panel tile P for mma.m16n8k16 (g = lane / 4, t = lane % 4): word 0 rows g,
+// columns 2t, 2t + 1; word 1 row g + 8; words 2, 3 the same rows, columns 2t + 8, 2t + 9.  As the A
+// operand (P itself) all four words are used; as the B operand (P^T) half h of the 8-wide column
+// blocks takes words h and h + 2.
+struct PanelFrag {
+  uint32_t w[3][4];
+};
+__device__ __forceinline__ void load_panel_frag(const float* __restrict__ Tt, int g, int t,
+                                                PanelFrag& f) {
+  const float2 v0 = *reinterpret_cast<const float2*>(Tt + elem_off(g, 2 * t));
+  const float2 v1 = *reinterpret_cast<const float2*>(Tt + elem_off(g + 8, 2 * t));
+  const float2 v2 = *reinterpret_cast<const float2*>(Tt + elem_off(g, 2 * t + 8));
+  const float2 v3 = *reinterpret_cast<const float2*>(Tt + elem_off(g + 8, 2 * t + 8));
+  split_pair(v0.x, v0.y, f.w[0][0], f.w[1][0], f.w[2][0]);
+  split_pair(v1.x, v1.y, f.w[0][1], f.w[1][1], f.w[2][1]);
+  split_pair(v2.x, v2.y, f.w[0][2], f.w[1][2], f.w[2][2]);
+  split_pair(v3.x, v3.y, f.w[0][3], f.w[1][3], f.w[2][3]);
+}
+
+// acc[h] += P_a P_b^T (the two 8-column halves h) from the six plane products, smallest first
+__device__ __forceinline__ void frag_product(float (&acc)[2][4], const PanelFrag& fa,
+                                             const PanelFrag& fb) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    mma_bf16_16816(acc[h], fa.w[1], fb.w[1][h], fb.w[1][h + 2]);  // m m
+    mma_bf16_16816(acc[h], fa.w[2], fb.w[0][h], fb.w[0][h + 2]);  // l h
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[2][h], fb.w[2][h + 2]);  // h l
+    mma_bf16_16816(acc[h], fa.w[1], fb.w[0][h], fb.w[0][h + 2]);  // m h
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[1][h], fb.w[1][h + 2]);  // h m
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[0][h], fb.w[0][h + 2]);  // h h
+  }
+}
+
+// C -= acc for one target tile (accumulator layout: rows g, g + 8, columns 8 h + 2 t, + 1)
+__device__ __forceinline__ void tile_subtract(float* __restrict__ Ct, const float (&acc)[2][4],
+                                              int g, int t) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float2* c0 = reinterpret_cast<float2*>(Ct + elem_off(g, 8 * h + 2 * t));
+    float2* c1 = reinterpret_cast<float2*>(Ct + elem_off(g + 8, 8 * h + 2 * t));
+    float2 u0 = *c0, u1 = *c1;
+    u0.x -= acc[h][0];
+    u0.y -= acc[h][1];
+    u1.x -= acc[h][2];
+    u1.y -= acc[h][3];
+    *c0 = u0;
+    *c1 = u1;
+  }
+}
+
+// Panel tile as a product: L_IK = A_IK L_KK^{-T} (fa: fragment of A_IK, fl: fragment of
+// L_KK^{-1}).  The result is stored over A_IK and returned as the fragment for the trailing
+// updates (the accumulator layout is the A-operand layout).
+__device__ __forceinline__ void panel_product(float* __restrict__ Tt, const PanelFrag& fa,
+                                              const PanelFrag& fl, int g, int t, PanelFrag& out) {
+  float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  frag_product(acc, fa, fl);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    *reinterpret_cast<float2*>(Tt + elem_off(g, 8 * h + 2 * t)) = make_float2(acc[h][0], acc[h][1]);
+    *reinterpret_cast<float2*>(Tt + elem_off(g + 8, 8 * h + 2 * t)) = make_float2(acc[h][2], acc[h][3]);
+    split_pair(acc[h][0], acc[h][1], out.w[0][2 * h], out.w[1][2 * h], out.w[2][2 * h]);
+    split_pair(acc[h][2], acc[h][3], out.w[0][2 * h + 1], out.w[1][2 * h + 1], out.w[2][2 * h + 1]);
+  }
+}
+
+// Cholesky of a diagonal tile together with the inverse of its factor.  Lanes 0..15 hold the rows
+// of A_KK, lanes 16..31 the rows of the identity; the column operations of the factorisation
+// (scale column j, subtract its multiples from the columns to the right) turn [A_KK; I] into
+// [L; L^{-T}].  Every lane also carries its own diagonal entry, so the pivot of the next column
+// does not wait for the updates of the others.  Stored: L in the lower triangle and diagonal of
+// the tile, the strict upper triangle of L^{-T} above it, 1 / l_jj (the diagonal of L^{-1}) in
+// invd.  Columns col0 + j >= n (identity padding) get pivot 1.  Returns the first column with a
+// pivot that is not positive, -1 if there is none.
+__device__ __forceinline__ int factor_diag_tile_inv(float* __restrict__ Tt, float* __restrict__ invd,
+                                                    int col0, int n, int lane) {
+  const int r = lane & 15;
+  const bool top = lane < 16;
+  float a[16];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float4 v = *reinterpret_cast<const float4*>(Tt + chunk_off(r, c));
+    a[4 * c] = v.x; a[4 * c + 1] = v.y; a[4 * c + 2] = v.z; a[4 * c + 3] = v.w;
+  }
+  float diag = 0.f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (r == j) diag = a[j];
+    if (!top) a[j] = (r == j) ? 1.f : 0.f;
+  }
+  int bad = -1;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    float dj = __shfl_sync(FULL, diag, j);
+    if (col0 + j < n) {
+      if (!(dj > 0.f) || !isfinite(dj)) {
+        if (bad < 0) bad = col0 + j;
+        dj = 1.f;
+      }
+    } else {
+      dj = 1.f;
+    }
+    const float rinv = rsqrtf(dj);
+    if (lane == 0) invd[col0 + j] = rinv;
+    a[j] *= rinv;
+    diag = fmaf(-a[j], a[j], diag);  // meaningful for the rows below j, whose pivots come later
+#pragma unroll
+    for (int v = j + 1; v < 16; ++v) {
+      const float lvj = __shfl_sync(FULL, a[j], v);
+      a[v] = fmaf(-a[j], lvj, a[v]);
+    }
+  }
+  // row r of the tile: columns <= r from the upper half-warp (L), columns > r from the lower
+  // half-warp (L^{-T})
+#pragma unroll
+  for (int cidx = 0; cidx < 16; ++cidx) {
+    if (top ? (cidx <= r) : (cidx > r)) Tt[elem_off(r, cidx)] = a[cidx];
+  }
+  __syncwarp();
+  return bad;
+}
+
+// Fragment of L_KK^{-1} (lower triangular) from a factored diagonal tile: entry (i, j), j < i, is
+// stored transposed at (j, i); the diagonal is invd.
+__device__ __forceinline__ void load_inverse_frag(const float* __restrict__ Tt,
+                                                  const float* __restrict__ invd16, int g, int t,
+                                                  PanelFrag& f) {
+  float v[4][2];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const int row = g + 8 * (w & 1);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int col = 2 * t + 8 * (w >> 1) + e;
+      float x = 0.f;
+      if (col < row) x = Tt[elem_off(col, row)];
+      else if (col == row) x = invd16[row];
+      v[w][e] = x;
+    }
+  }
+#pragma unroll
+  for (int w = 0; w < 4; ++w) split_pair(v[w][0], v[w][1], f.w[0][w], f.w[1][w], f.w[2][w]);
+}
+
+// One warp per row; the arguments and the split of the CTAs between the two kinds of rows are
+// those of solve_rows_fast_kernel (solve.cu).  `tiles` is the number of tile rows the launch
+// provides room for; a row uses ceil(n / 16) of them.
+__global__ void __launch_bounds__(32 * 16)
+solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
+                       const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
+                       __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
+                       int ldd, int tiles, int mat_in_smem, const int* __restrict__ row_lists,
+                       const unsigned* __restrict__ list_counts, int fixed_kind, int report_max_s,
+                       thanos_stats_t* stats) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int warps = blockDim.x >> 5;
+  const TileSolveLayout lay = tile_solve_layout(Bw, tiles, mat_in_smem != 0);
+  float* Ms = reinterpret_cast<float*>(dyn);
+  unsigned char* wbase = dyn + 4 * (size_t)lay.mat_floats + (size_t)warp * lay.per_warp_bytes;
+  float* A = reinterpret_cast<float*>(wbase);
+  float* invd = A + lay.tiles_floats;
+  float* yv = invd + 16 * tiles;
+  float* wblk = yv + 16 * tiles + 16;
+  float* dvec = wblk + Bw;
+  unsigned short* qlist = reinterpret_cast<unsigned short*>(dvec + Bw);
+  unsigned short* klist = qlist + Bw + 16;
+  const int g = lane >> 2, t4 = lane & 3;
+
+  int cnt[2];
+  if (row_lists) {
+    cnt[0] = (int)list_counts[0];
+    cnt[1] = (int)list_counts[1];
+  } else {
+    cnt[fixed_kind] = c;
+    cnt[fixed_kind ^ 1] = 0;
+  }
+  const int nctas = gridDim.x;
+  int n1 = 0;  // CTAs [0, nctas - n1) serve kind 0, the rest kind 1
+  if (cnt[1] > 0) {
+    if (cnt[0] == 0) {
+      n1 = nctas;
+    } else {
+      n1 = (int)(((long long)nctas * cnt[1] + (cnt[0] + cnt[1]) / 2) / (cnt[0] + cnt[1]));
+      if (n1 < 1) n1 = 1;
+      if (n1 > nctas - 1) n1 = nctas - 1;
+    }
+  }
+  const bool both_here = nctas == 1 && cnt[0] > 0 && cnt[1] > 0;
+  const unsigned lt = (1u << lane) - 1u;
+
+  for (int pass = 0; pass < (both_here ? 2 : 1); ++pass) {
+    int kind, my_index, my_ctas;
+    if (both_here) {
+      kind = pass;
+      my_index = 0;
+      my_ctas = 1;
+    } else if ((int)blockIdx.x < nctas - n1) {
+      kind = 0;
+      my_index = blockIdx.x;
+      my_ctas = nctas - n1;
+    } else {
+      kind = 1;
+      my_index = blockIdx.x - (nctas - n1);
+      my_ctas = n1;
+    }
+    if (cnt[kind] == 0) continue;  // CTA-uniform
+    const bool kpath = kind == 1;
+    const float* Mat = kpath ? Sm : Gm;
+    const float* M;
+    int ldm;
+    if (mat_in_smem) {
+      __syncthreads();
+      const int q4 = Bw >> 2;
+      for (int i = warp; i < Bw; i += warps) {
+        const float4* src = reinterpret_cast<const float4*>(Mat + (int64_t)i * ld_mat);
+        for (int j = lane; j < q4; j += 32) {
+          const float4 v = src[j];
+          float* dst = Ms + i * lay.ldm + 4 * j;
+          dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+        }
+      }
+      __syncthreads();
+      M = Ms;
+      ldm = lay.ldm;
+    } else {
+      M = Mat;
+      ldm = ld_mat;
+    }
+    const int* rlist = row_lists ? row_lists + (size_t)kind * c : nullptr;
+
+    for (int li = my_index * warps + warp; li < cnt[kind]; li += my_ctas * warps) {
+      const int row = rlist ? rlist[li] : li;
+      const uint8_t* mrow = mask + (int64_t)row * b + j1;
+      float* wrow = Wc + (int64_t)row * b + j1;
+      // ---- q = phi(mask row) and its complement k, both ascending
+      int s = 0, t = 0;
+      for (int base = 0; base < Bw; base += 128) {
+        uint8_t mv[4];
+        float wv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int jj = base + 32 * u + lane;
+          mv[u] = (jj < Bw) ? mrow[jj] : (uint8_t)2;
+          wv[u] = (jj < Bw) ? wrow[jj] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int jj = base + 32 * u + lane;
+          const bool mb = mv[u] == 1;
+          const bool kb = mv[u] == 0;
+          const unsigned bq = __ballot_sync(FULL, mb);
+          const unsigned bk = __ballot_sync(FULL, kb);
+          if (mb) qlist[s + __popc(bq & lt)] = (unsigned short)jj;
+          if (kb) klist[t + __popc(bk & lt)] = (unsigned short)jj;
+          if (jj < Bw) wblk[jj] = wv[u];
+          s += __popc(bq);
+          t += __popc(bk);
+        }
+      }
+      if (s == 0) {  // nothing removed: the row is not touched in this block
+        for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+        __syncwarp();
+        continue;
+      }
+      if (report_max_s && row == 0 && lane == 0) atomicMax(&stats->max_s, s);
+      const int n = kpath ? t : s;    // unknowns of this row's system
+      const int no = kpath ? s : t;   // size of the other set
+      unsigned short* sel = kpath ? klist : qlist;
+      unsigned short* oth = kpath ? qlist : klist;
+      if (lane < 16) {
+        sel[n + lane] = 0;
+        oth[no + lane] = 0;
+      }
+      const int T = (n + 15) >> 4;
+      if (n == 0) {  // every weight of the block is removed: delta = -w, nothing to solve
+        for (int jj = lane; jj < Bw; jj += 32) {
+          const float d = -wblk[jj];
+          wrow[jj] = 0.f;
+          store_split3(D + (int64_t)row * ldd + jj, dplane, d);
+        }
+        __syncwarp();
+        continue;
+      }
+      if ((s > t) != kpath || T > tiles) {
+        // cannot happen for lists and launch sizes made by this library
+        if (lane == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
+        __syncwarp();
+        continue;
+      }
+      __syncwarp();
+      // ---- right-hand side: w_q (direct form) or g_e = sum_a w[q_a] S[q_a, k_e] (complement),
+      //      zero beyond n
+      for (int e0 = 0; e0 < 16 * T; e0 += 32) {
+        const int e = e0 + lane;
+        float gsum = 0.f;
+        if (!kpath) {
+          if (e < n) gsum = wblk[sel[e]];
+        } else {
+          const int col = (e < n) ? (int)sel[e] : 0;
+          float g0 = 0.f, g1 = 0.f;
+          for (int a = 0; a < no; a += 4) {
+            const ushort4 ix = *reinterpret_cast<const ushort4*>(oth + a);
+            const float w0 = wblk[ix.x];
+            const float w1 = (a + 1 < no) ? wblk[ix.y] : 0.f;
+            const float w2 = (a + 2 < no) ? wblk[ix.z] : 0.f;
+            const float w3 = (a + 3 < no) ? wblk[ix.w] : 0.f;
+            g0 = fmaf(w0, M[(int)ix.x * ldm + col], g0);
+            g1 = fmaf(w1, M[(int)ix.y * ldm + col], g1);
+            g0 = fmaf(w2, M[(int)ix.z * ldm + col], g0);
+            g1 = fmaf(w3, M[(int)ix.w * ldm + col], g1);
+          }
+          gsum = e < n ? g0 + g1 : 0.f;
+        }
+        if (e < 16 * T) yv[e] = gsum;
+      }
+      // ---- gather the lower triangle of M[sel, sel] into tiles, identity beyond n: lane
+      //      (r0 = lane / 16, k = lane % 16) fills rows r0 + 2 h of column k of every tile
+      {
+        const int r0 = lane >> 4, k = lane & 15;
+        for (int I = 0; I < T; ++I) {
+          int rowoff[8];
+#pragma unroll
+          for (int h = 0; h < 8; ++h) {
+            const int i = 16 * I + r0 + 2 * h;
+            rowoff[h] = i < n ? (int)sel[i] * ldm : -1;
+          }
+          for (int J = 0; J <= I; ++J) {
+            const int j = 16 * J + k;
+            const int cj = j < n ? (int)sel[j] : -1;
+            float v[8];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+              const int i = 16 * I + r0 + 2 * h;
+              v[h] = (rowoff[h] >= 0 && cj >= 0) ? M[rowoff[h] + cj] : (i == j ? 1.f : 0.f);
+            }
+            float* Tt = A + tbase(I, J);
+#pragma unroll
+            for (int h = 0; h < 8; ++h) Tt[elem_off(r0 + 2 * h, k)] = v[h];
+          }
+        }
+      }
+      __syncwarp();
+
+      // ---- right-looking tile Cholesky
+      bool bad = false;
+      for (int K = 0; K < T; ++K) {
+        float* Lk = A + tbase(K, K);
+        bad |= factor_diag_tile_inv(Lk, invd, 16 * K, n, lane) >= 0;
+        const int m = T - K - 1;  // tile rows below the diagonal tile (warp-uniform, <= 3)
+        if (m == 0) break;
+        // panel tiles as products with the inverse of the diagonal factor
+        PanelFrag fl, f0, f1, f2;
+        load_inverse_frag(Lk, invd + 16 * K, g, t4, fl);
+        {
+          PanelFrag fa;
+          load_panel_frag(A + tbase(K + 1, K), g, t4, fa);
+          panel_product(A + tbase(K + 1, K), fa, fl, g, t4, f0);
+          if (m > 1) {
+            load_panel_frag(A + tbase(K + 2, K), g, t4, fa);
+            panel_product(A + tbase(K + 2, K), fa, fl, g, t4, f1);
+          }
+          if (m > 2) {
+            load_panel_frag(A + tbase(K + 3, K), g, t4, fa);
+            panel_product(A + tbase(K + 3, K), fa, fl, g, t4, f2);
+          }
+        }
+        // trailing tiles, one tile row at a time (its products are independent chains)
+        {
+          float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          frag_product(acc, f0, f0);
+          tile_subtract(A + tbase(K + 1, K + 1), acc, g, t4);
+        }
+        if (m > 1) {
+          float a0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          float a1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          frag_product(a0, f1, f0);
+          frag_product(a1, f1, f1);
+          tile_subtract(A + tbase(K + 2, K + 1), a0, g, t4);
+          tile_subtract(A + tbase(K + 2, K + 2), a1, g, t4);
+        }
+        if (m > 2) {
+          float a0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          float a1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          float a2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+          frag_product(a0, f2, f0);
+          frag_product(a1, f2, f1);
+          frag_product(a2, f2, f2);
+          tile_subtract(A + tbase(K + 3, K + 1), a0, g, t4);
+          tile_subtract(A + tbase(K + 3, K + 2), a1, g, t4);
+          tile_subtract(A + tbase(K + 3, K + 3), a2, g, t4);
+        }
+        __syncwarp();
+      }
+      if (bad) {
+        if (lane == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
+        for (int jj = lane; jj < Bw; jj += 32) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
+        __syncwarp();
+        continue;
+      }
+
+      const int l16 = lane & 15, hh = lane >> 4;
+      // ---- forward substitution L y = rhs by tile rows: y_I = L_II^{-1} (rhs_I - sum_J L_IJ y_J);
+      //      lanes l and l + 16 share row l (columns 0..7 and 8..15 of every tile)
+      for (int I = 0; I < T; ++I) {
+        if (I > 0) {
+          float acc = 0.f;
+          for (int J = 0; J < I; ++J) {
+            const float* Lt = A + tbase(I, J);
+            const float4 a0 = *reinterpret_cast<const float4*>(Lt + chunk_off(l16, 2 * hh));
+            const float4 a1 = *reinterpret_cast<const float4*>(Lt + chunk_off(l16, 2 * hh + 1));
+            const float4 y0 = *reinterpret_cast<const float4*>(yv + 16 * J + 8 * hh);
+            const float4 y1 = *reinterpret_cast<const float4*>(yv + 16 * J + 8 * hh + 4);
+            acc = fmaf(a0.x, y0.x, acc); acc = fmaf(a0.y, y0.y, acc);
+            acc = fmaf(a0.z, y0.z, acc); acc = fmaf(a0.w, y0.w, acc);
+            acc = fmaf(a1.x, y1.x, acc); acc = fmaf(a1.y, y1.y, acc);
+            acc = fmaf(a1.z, y1.z, acc); acc = fmaf(a1.w, y1.w, acc);
+          }
+          acc += __shfl_xor_sync(FULL, acc, 16);
+          __syncwarp();
+          if (lane < 16) yv[16 * I + lane] -= acc;
+          __syncwarp();
+        }
+        // y = L_II^{-1} v: entry (l, c), c < l, of the inverse sits at (c, l) of the tile
+        const float* Lk = A + tbase(I, I);
+        const float4 v0 = *reinterpret_cast<const float4*>(yv + 16 * I + 8 * hh);
+        const float4 v1 = *reinterpret_cast<const float4*>(yv + 16 * I + 8 * hh + 4);
+        const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int cidx = 8 * hh + e;
+          const float x = cidx < l16 ? Lk[elem_off(cidx, l16)] : (cidx == l16 ? invd[16 * I + l16] : 0.f);
+          acc = fmaf(x, vv[e], acc);
+        }
+        acc += __shfl_xor_sync(FULL, acc, 16);
+        __syncwarp();
+        if (lane < 16) yv[16 * I + lane] = acc;
+        __syncwarp();
+      }
+      // ---- back substitution L^T x = y from the bottom: x_K = L_KK^{-T} y_K, then the rows above
+      //      lose L_KJ^T x_K
+      for (int Kb = T - 1; Kb >= 0; --Kb) {
+        const float* Lk = A + tbase(Kb, Kb);
+        {
+          // row l of L^{-T}: columns > l in the tile's upper triangle, the diagonal in invd
+          const float4 a0 = *reinterpret_cast<const float4*>(Lk + chunk_off(l16, 2 * hh));
+          const float4 a1 = *reinterpret_cast<const float4*>(Lk + chunk_off(l16, 2 * hh + 1));
+          const float4 v0 = *reinterpret_cast<const float4*>(yv + 16 * Kb + 8 * hh);
+          const float4 v1 = *reinterpret_cast<const float4*>(yv + 16 * Kb + 8 * hh + 4);
+          const float aa[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+          const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          const float dl = invd[16 * Kb + l16];
+          float acc = 0.f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int cidx = 8 * hh + e;
+            const float x = cidx > l16 ? aa[e] : (cidx == l16 ? dl : 0.f);
+            acc = fmaf(x, vv[e], acc);
+          }
+          acc += __shfl_xor_sync(FULL, acc, 16);
+          __syncwarp();
+          if (lane < 16) yv[16 * Kb + lane] = acc;
+          __syncwarp();
+        }
+        // earlier unknowns: y_k -= sum_w L[16 Kb + w][k] x_w
+        for (int k = lane; k < 16 * Kb; k += 32) {
+          const float* Lt = A + tbase(Kb, k >> 4);
+          const int kk = k & 15;
+          float acc = 0.f;
+#pragma unroll
+          for (int w = 0; w < 16; ++w) acc = fmaf(Lt[elem_off(w, kk)], yv[16 * Kb + w], acc);
+          yv[k] -= acc;
+        }
+        __syncwarp();
+      }
+
+      // ---- delta over the block
+      for (int a = lane; a < s; a += 32) dvec[qlist[a]] = -wblk[qlist[a]];
+      if (kpath) {
+        for (int e = lane; e < n; e += 32) dvec[sel[e]] = yv[e];
+      } else {
+        // delta_k = -sum_a lambda_a G[q_a, k_e]   (yv is zero beyond n)
+        for (int e0 = 0; e0 < no; e0 += 32) {
+          const int e = e0 + lane;
+          const int col = (e < no) ? (int)oth[e] : 0;
+          float g0 = 0.f, g1 = 0.f;
+          for (int a = 0; a < n; a += 4) {
+            const ushort4 ix = *reinterpret_cast<const ushort4*>(sel + a);
+            const float4 xv = *reinterpret_cast<const float4*>(yv + a);
+            g0 = fmaf(xv.x, M[(int)ix.x * ldm + col], g0);
+            g1 = fmaf(xv.y, M[(int)ix.y * ldm + col], g1);
+            g0 = fmaf(xv.z, M[(int)ix.z * ldm + col], g0);
+            g1 = fmaf(xv.w, M[(int)ix.w * ldm + col], g1);
+          }
+          if (e < no) dvec[col] = -(g0 + g1);
+        }
+      }
+      __syncwarp();
+      for (int jj = lane; jj < Bw; jj += 32) {
+        const float d = dvec[jj];
+        const bool removed = mrow[jj] != 0;
+        wrow[jj] = removed ? 0.f : wblk[jj] + d;
+        store_split3(D + (int64_t)row * ldd + jj, dplane, d);
+      }
+      __syncwarp();
+    }
+  }
+}
+
+constexpr size_t TILE_SMEM_BUDGET = 227 * 1024;
+constexpr int TILE_MAX_WARPS = 16;
+constexpr float TILE_UNCACHED_ROW_COST = 1.2f;  // time of a row without the shared copy of G / S over with it (measured: 63 k against 53 k cycles)
+
+}  // namespace
+
+int tile_solve_max_unknowns() { return 16 * TILE_T_MAX; }
+
+// Same contract as launch_fast of solve.cu; n_max <= 64.
+thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G, const float* S,
+                                  int ld_mat, __nv_bfloat16* D, int64_t dplane, int c, int b,
+                                  int j1, int Bw, int ldd, int n_max, const int* row_lists,
+                                  const unsigned* list_counts, int fixed_kind, int report_max_s,
+                                  thanos_stats_t* stats, cudaStream_t stream) {
+  const int T = (n_max + 15) / 16 < 1 ? 1 : (n_max + 15) / 16;
+  if (T > TILE_T_MAX) return THANOS_ERR_SHAPE;
+  // a launch lasts (rows per warp, rounded up) x (time of a row): with the shared copy of G / S a
+  // row is faster, without it more warps fit -- take whichever product is smaller
+  const bool can_copy = (size_t)Bw * (Bw | 1) * 4 <= 72 * 1024;
+  bool in_smem = false;
+  int warps = 0;
+  float best = 0.f;
+  for (int copy = can_copy ? 1 : 0; copy >= 0; --copy) {
+    const TileSolveLayout l = tile_solve_layout(Bw, T, copy != 0);
+    int wmax = (int)((TILE_SMEM_BUDGET - 4 * (size_t)l.mat_floats) / l.per_warp_bytes);
+    if (wmax > TILE_MAX_WARPS) wmax = TILE_MAX_WARPS;
+    for (int w = wmax; w >= 1 && w >= wmax - 1; --w) {
+      const float cost =
+          (float)ceil_div(c, (int64_t)NUM_SMS * w) * (copy ? 1.f : TILE_UNCACHED_ROW_COST);
+      if (warps == 0 || cost < best) {
+        best = cost;
+        warps = w;
+        in_smem = copy != 0;
+      }
+    }
+  }
+  if (warps < 1) return THANOS_ERR_SHAPE;
+  const TileSolveLayout lay = tile_solve_layout(Bw, T, in_smem);
+  const size_t smem = 4 * (size_t)lay.mat_floats + (size_t)warps * lay.per_warp_bytes;
+  {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_tile_kernel, (int)TILE_SMEM_BUDGET, done));
+  }
+  int64_t grid = ceil_div(c, warps);
+  if (grid > NUM_SMS) grid = NUM_SMS;
+  solve_rows_tile_kernel<<<(unsigned)grid, warps * 32, smem, stream>>>(
+      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, T, in_smem ? 1 : 0, row_lists,
+      list_counts, fixed_kind, report_max_s, stats);
+  THANOS_CHECK_LAUNCH();
+  return THANOS_OK;
+}
+
+}  // namespace thanos
