@@ -31,16 +31,12 @@ constexpr int TILE_T_MAX = 4;  // tile rows: systems of up to 64 unknowns
 __device__ __forceinline__ int tbase(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
 
 struct TileSolveLayout {
-  int mat_floats;      // shared copy of G or S (0 when it stays in global memory)
-  int ldm;
   int tiles_floats;
   int per_warp_bytes;
 };
 
-__host__ __device__ inline TileSolveLayout tile_solve_layout(int Bw, int T, bool mat_in_smem) {
+__host__ __device__ inline TileSolveLayout tile_solve_layout(int Bw, int T) {
   TileSolveLayout L;
-  L.ldm = mat_in_smem ? (Bw | 1) : 0;
-  L.mat_floats = mat_in_smem ? ((Bw * L.ldm + 3) & ~3) : 0;
   L.tiles_floats = (T * (T + 1) / 2) * 256;
   // tiles, invd[16 T], yv[16 T + 16], wblk[Bw], dvec[Bw], two index lists of Bw + 16 shorts
   const int bytes = 4 * (L.tiles_floats + 16 * T + 16 * T + 16 + 2 * Bw) + 2 * 2 * (Bw + 16);
@@ -79,12 +75,26 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& p0, uin
 struct PanelFrag {
   uint32_t w[3][4];
 };
-__device__ __forceinline__ void load_panel_frag(const float* __restrict__ Tt, int g, int t,
+// Offsets of a lane's four fragment words inside any tile (they depend on the lane only): word
+// 2 h' + h'' is row g + 8 h'', columns 2t + 8 h' -- also the lane's accumulator entries of column
+// half h'.
+struct FragOff {
+  int o[4];
+};
+__device__ __forceinline__ FragOff make_frag_off(int g, int t) {
+  FragOff f;
+  f.o[0] = elem_off(g, 2 * t);
+  f.o[1] = elem_off(g + 8, 2 * t);
+  f.o[2] = elem_off(g, 2 * t + 8);
+  f.o[3] = elem_off(g + 8, 2 * t + 8);
+  return f;
+}
+__device__ __forceinline__ void load_panel_frag(const float* __restrict__ Tt, const FragOff& fo,
                                                 PanelFrag& f) {
-  const float2 v0 = *reinterpret_cast<const float2*>(Tt + elem_off(g, 2 * t));
-  const float2 v1 = *reinterpret_cast<const float2*>(Tt + elem_off(g + 8, 2 * t));
-  const float2 v2 = *reinterpret_cast<const float2*>(Tt + elem_off(g, 2 * t + 8));
-  const float2 v3 = *reinterpret_cast<const float2*>(Tt + elem_off(g + 8, 2 * t + 8));
+  const float2 v0 = *reinterpret_cast<const float2*>(Tt + fo.o[0]);
+  const float2 v1 = *reinterpret_cast<const float2*>(Tt + fo.o[1]);
+  const float2 v2 = *reinterpret_cast<const float2*>(Tt + fo.o[2]);
+  const float2 v3 = *reinterpret_cast<const float2*>(Tt + fo.o[3]);
   split_pair(v0.x, v0.y, f.w[0][0], f.w[1][0], f.w[2][0]);
   split_pair(v1.x, v1.y, f.w[0][1], f.w[1][1], f.w[2][1]);
   split_pair(v2.x, v2.y, f.w[0][2], f.w[1][2], f.w[2][2]);
@@ -107,11 +117,11 @@ __device__ __forceinline__ void frag_product(float (&acc)[2][4], const PanelFrag
 
 // C -= acc for one target tile (accumulator layout: rows g, g + 8, columns 8 h + 2 t, + 1)
 __device__ __forceinline__ void tile_subtract(float* __restrict__ Ct, const float (&acc)[2][4],
-                                              int g, int t) {
+                                              const FragOff& fo) {
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    float2* c0 = reinterpret_cast<float2*>(Ct + elem_off(g, 8 * h + 2 * t));
-    float2* c1 = reinterpret_cast<float2*>(Ct + elem_off(g + 8, 8 * h + 2 * t));
+    float2* c0 = reinterpret_cast<float2*>(Ct + fo.o[2 * h]);
+    float2* c1 = reinterpret_cast<float2*>(Ct + fo.o[2 * h + 1]);
     float2 u0 = *c0, u1 = *c1;
     u0.x -= acc[h][0];
     u0.y -= acc[h][1];
@@ -126,13 +136,14 @@ __device__ __forceinline__ void tile_subtract(float* __restrict__ Ct, const floa
 // L_KK^{-1}).  The result is stored over A_IK and returned as the fragment for the trailing
 // updates (the accumulator layout is the A-operand layout).
 __device__ __forceinline__ void panel_product(float* __restrict__ Tt, const PanelFrag& fa,
-                                              const PanelFrag& fl, int g, int t, PanelFrag& out) {
+                                              const PanelFrag& fl, const FragOff& fo,
+                                              PanelFrag& out) {
   float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
   frag_product(acc, fa, fl);
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    *reinterpret_cast<float2*>(Tt + elem_off(g, 8 * h + 2 * t)) = make_float2(acc[h][0], acc[h][1]);
-    *reinterpret_cast<float2*>(Tt + elem_off(g + 8, 8 * h + 2 * t)) = make_float2(acc[h][2], acc[h][3]);
+    *reinterpret_cast<float2*>(Tt + fo.o[2 * h]) = make_float2(acc[h][0], acc[h][1]);
+    *reinterpret_cast<float2*>(Tt + fo.o[2 * h + 1]) = make_float2(acc[h][2], acc[h][3]);
     split_pair(acc[h][0], acc[h][1], out.w[0][2 * h], out.w[1][2 * h], out.w[2][2 * h]);
     split_pair(acc[h][2], acc[h][3], out.w[0][2 * h + 1], out.w[1][2 * h + 1], out.w[2][2 * h + 1]);
   }
@@ -223,16 +234,15 @@ __global__ void __launch_bounds__(32 * 16)
 solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                        const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
                        __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
-                       int ldd, int tiles, int mat_in_smem, const int* __restrict__ row_lists,
+                       int ldd, int tiles, const int* __restrict__ row_lists,
                        const unsigned* __restrict__ list_counts, int fixed_kind, int report_max_s,
                        thanos_stats_t* stats) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int warps = blockDim.x >> 5;
-  const TileSolveLayout lay = tile_solve_layout(Bw, tiles, mat_in_smem != 0);
-  float* Ms = reinterpret_cast<float*>(dyn);
-  unsigned char* wbase = dyn + 4 * (size_t)lay.mat_floats + (size_t)warp * lay.per_warp_bytes;
+  const TileSolveLayout lay = tile_solve_layout(Bw, tiles);
+  unsigned char* wbase = dyn + (size_t)warp * lay.per_warp_bytes;
   float* A = reinterpret_cast<float*>(wbase);
   float* invd = A + lay.tiles_floats;
   float* yv = invd + 16 * tiles;
@@ -241,6 +251,11 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   unsigned short* qlist = reinterpret_cast<unsigned short*>(dvec + Bw);
   unsigned short* klist = qlist + Bw + 16;
   const int g = lane >> 2, t4 = lane & 3;
+  const FragOff fo = make_frag_off(g, t4);
+  // gather: lane (r0 = lane / 16, k = lane % 16) fills rows r0 + 2 h of column k of a tile
+  int gofs[8];
+#pragma unroll
+  for (int h = 0; h < 8; ++h) gofs[h] = elem_off((lane >> 4) + 2 * h, lane & 15);
 
   int cnt[2];
   if (row_lists) {
@@ -281,27 +296,10 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     }
     if (cnt[kind] == 0) continue;  // CTA-uniform
     const bool kpath = kind == 1;
-    const float* Mat = kpath ? Sm : Gm;
-    const float* M;
-    int ldm;
-    if (mat_in_smem) {
-      __syncthreads();
-      const int q4 = Bw >> 2;
-      for (int i = warp; i < Bw; i += warps) {
-        const float4* src = reinterpret_cast<const float4*>(Mat + (int64_t)i * ld_mat);
-        for (int j = lane; j < q4; j += 32) {
-          const float4 v = src[j];
-          float* dst = Ms + i * lay.ldm + 4 * j;
-          dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
-        }
-      }
-      __syncthreads();
-      M = Ms;
-      ldm = lay.ldm;
-    } else {
-      M = Mat;
-      ldm = ld_mat;
-    }
+    // G / S are read from global memory (64 KB at B = 128: they stay in L2); a shared copy
+    // would cost three of sixteen warps and buys no throughput
+    const float* M = kpath ? Sm : Gm;
+    const int ldm = ld_mat;
     const int* rlist = row_lists ? row_lists + (size_t)kind * c : nullptr;
 
     for (int li = my_index * warps + warp; li < cnt[kind]; li += my_ctas * warps) {
@@ -366,52 +364,57 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       __syncwarp();
       // ---- right-hand side: w_q (direct form) or g_e = sum_a w[q_a] S[q_a, k_e] (complement),
       //      zero beyond n
-      for (int e0 = 0; e0 < 16 * T; e0 += 32) {
-        const int e = e0 + lane;
-        float gsum = 0.f;
-        if (!kpath) {
-          if (e < n) gsum = wblk[sel[e]];
-        } else {
+      if (!kpath) {
+        for (int e = lane; e < 16 * T; e += 32) yv[e] = e < n ? wblk[sel[e]] : 0.f;
+      } else {
+        // the removed weights in list order, zero-padded to a multiple of four
+        for (int a = lane; a < ((no + 3) & ~3); a += 32) dvec[a] = a < no ? wblk[oth[a]] : 0.f;
+        __syncwarp();
+        for (int e0 = 0; e0 < 16 * T; e0 += 32) {
+          const int e = e0 + lane;
           const int col = (e < n) ? (int)sel[e] : 0;
           float g0 = 0.f, g1 = 0.f;
           for (int a = 0; a < no; a += 4) {
             const ushort4 ix = *reinterpret_cast<const ushort4*>(oth + a);
-            const float w0 = wblk[ix.x];
-            const float w1 = (a + 1 < no) ? wblk[ix.y] : 0.f;
-            const float w2 = (a + 2 < no) ? wblk[ix.z] : 0.f;
-            const float w3 = (a + 3 < no) ? wblk[ix.w] : 0.f;
-            g0 = fmaf(w0, M[(int)ix.x * ldm + col], g0);
-            g1 = fmaf(w1, M[(int)ix.y * ldm + col], g1);
-            g0 = fmaf(w2, M[(int)ix.z * ldm + col], g0);
-            g1 = fmaf(w3, M[(int)ix.w * ldm + col], g1);
+            const float4 wq = *reinterpret_cast<const float4*>(dvec + a);
+            g0 = fmaf(wq.x, M[(int)ix.x * ldm + col], g0);
+            g1 = fmaf(wq.y, M[(int)ix.y * ldm + col], g1);
+            g0 = fmaf(wq.z, M[(int)ix.z * ldm + col], g0);
+            g1 = fmaf(wq.w, M[(int)ix.w * ldm + col], g1);
           }
-          gsum = e < n ? g0 + g1 : 0.f;
+          if (e < 16 * T) yv[e] = e < n ? g0 + g1 : 0.f;
         }
-        if (e < 16 * T) yv[e] = gsum;
+        __syncwarp();
       }
-      // ---- gather the lower triangle of M[sel, sel] into tiles, identity beyond n: lane
-      //      (r0 = lane / 16, k = lane % 16) fills rows r0 + 2 h of column k of every tile
+      // ---- gather the lower triangle of M[sel, sel] into tiles, identity beyond n
       {
         const int r0 = lane >> 4, k = lane & 15;
         for (int I = 0; I < T; ++I) {
+          const bool rows_in = 16 * I + 16 <= n;  // warp-uniform: every row of the tile row exists
           int rowoff[8];
 #pragma unroll
           for (int h = 0; h < 8; ++h) {
             const int i = 16 * I + r0 + 2 * h;
-            rowoff[h] = i < n ? (int)sel[i] * ldm : -1;
+            rowoff[h] = (rows_in || i < n) ? (int)sel[i] * ldm : -1;
           }
           for (int J = 0; J <= I; ++J) {
             const int j = 16 * J + k;
-            const int cj = j < n ? (int)sel[j] : -1;
-            float v[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-              const int i = 16 * I + r0 + 2 * h;
-              v[h] = (rowoff[h] >= 0 && cj >= 0) ? M[rowoff[h] + cj] : (i == j ? 1.f : 0.f);
-            }
             float* Tt = A + tbase(I, J);
+            float v[8];
+            if (rows_in) {  // columns j <= i < n as well
+              const float* Mc = M + (int)sel[j];
 #pragma unroll
-            for (int h = 0; h < 8; ++h) Tt[elem_off(r0 + 2 * h, k)] = v[h];
+              for (int h = 0; h < 8; ++h) v[h] = Mc[rowoff[h]];
+            } else {
+              const int cj = j < n ? (int)sel[j] : -1;
+#pragma unroll
+              for (int h = 0; h < 8; ++h) {
+                const int i = 16 * I + r0 + 2 * h;
+                v[h] = (rowoff[h] >= 0 && cj >= 0) ? M[rowoff[h] + cj] : (i == j ? 1.f : 0.f);
+              }
+            }
+#pragma unroll
+            for (int h = 0; h < 8; ++h) Tt[gofs[h]] = v[h];
           }
         }
       }
@@ -429,30 +432,30 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         load_inverse_frag(Lk, invd + 16 * K, g, t4, fl);
         {
           PanelFrag fa;
-          load_panel_frag(A + tbase(K + 1, K), g, t4, fa);
-          panel_product(A + tbase(K + 1, K), fa, fl, g, t4, f0);
+          load_panel_frag(A + tbase(K + 1, K), fo, fa);
+          panel_product(A + tbase(K + 1, K), fa, fl, fo, f0);
           if (m > 1) {
-            load_panel_frag(A + tbase(K + 2, K), g, t4, fa);
-            panel_product(A + tbase(K + 2, K), fa, fl, g, t4, f1);
+            load_panel_frag(A + tbase(K + 2, K), fo, fa);
+            panel_product(A + tbase(K + 2, K), fa, fl, fo, f1);
           }
           if (m > 2) {
-            load_panel_frag(A + tbase(K + 3, K), g, t4, fa);
-            panel_product(A + tbase(K + 3, K), fa, fl, g, t4, f2);
+            load_panel_frag(A + tbase(K + 3, K), fo, fa);
+            panel_product(A + tbase(K + 3, K), fa, fl, fo, f2);
           }
         }
         // trailing tiles, one tile row at a time (its products are independent chains)
         {
           float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
           frag_product(acc, f0, f0);
-          tile_subtract(A + tbase(K + 1, K + 1), acc, g, t4);
+          tile_subtract(A + tbase(K + 1, K + 1), acc, fo);
         }
         if (m > 1) {
           float a0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
           float a1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
           frag_product(a0, f1, f0);
           frag_product(a1, f1, f1);
-          tile_subtract(A + tbase(K + 2, K + 1), a0, g, t4);
-          tile_subtract(A + tbase(K + 2, K + 2), a1, g, t4);
+          tile_subtract(A + tbase(K + 2, K + 1), a0, fo);
+          tile_subtract(A + tbase(K + 2, K + 2), a1, fo);
         }
         if (m > 2) {
           float a0[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -461,9 +464,9 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           frag_product(a0, f2, f0);
           frag_product(a1, f2, f1);
           frag_product(a2, f2, f2);
-          tile_subtract(A + tbase(K + 3, K + 1), a0, g, t4);
-          tile_subtract(A + tbase(K + 3, K + 2), a1, g, t4);
-          tile_subtract(A + tbase(K + 3, K + 3), a2, g, t4);
+          tile_subtract(A + tbase(K + 3, K + 1), a0, fo);
+          tile_subtract(A + tbase(K + 3, K + 2), a1, fo);
+          tile_subtract(A + tbase(K + 3, K + 3), a2, fo);
         }
         __syncwarp();
       }
@@ -585,7 +588,6 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
 
 constexpr size_t TILE_SMEM_BUDGET = 227 * 1024;
 constexpr int TILE_MAX_WARPS = 16;
-constexpr float TILE_UNCACHED_ROW_COST = 1.2f;  // time of a row without the shared copy of G / S over with it (measured: 63 k against 53 k cycles)
 
 }  // namespace
 
@@ -599,29 +601,27 @@ thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G
                                   thanos_stats_t* stats, cudaStream_t stream) {
   const int T = (n_max + 15) / 16 < 1 ? 1 : (n_max + 15) / 16;
   if (T > TILE_T_MAX) return THANOS_ERR_SHAPE;
-  // a launch lasts (rows per warp, rounded up) x (time of a row): with the shared copy of G / S a
-  // row is faster, without it more warps fit -- take whichever product is smaller
-  const bool can_copy = (size_t)Bw * (Bw | 1) * 4 <= 72 * 1024;
-  bool in_smem = false;
+  // The kernel is bound by instruction issue, not by latency: an SM finishes a row every ~3.9 k
+  // cycles whether 13, 16 or 18 warps share it (measured), so a row takes (warps) x 3.9 k cycles and
+  // a launch lasts (rows per warp, rounded up) x (warps).  Pick the warp count that wastes the
+  // least of the last round.
   int warps = 0;
-  float best = 0.f;
-  for (int copy = can_copy ? 1 : 0; copy >= 0; --copy) {
-    const TileSolveLayout l = tile_solve_layout(Bw, T, copy != 0);
-    int wmax = (int)((TILE_SMEM_BUDGET - 4 * (size_t)l.mat_floats) / l.per_warp_bytes);
+  long long best = 0;
+  {
+    const TileSolveLayout l = tile_solve_layout(Bw, T);
+    int wmax = (int)(TILE_SMEM_BUDGET / l.per_warp_bytes);
     if (wmax > TILE_MAX_WARPS) wmax = TILE_MAX_WARPS;
-    for (int w = wmax; w >= 1 && w >= wmax - 1; --w) {
-      const float cost =
-          (float)ceil_div(c, (int64_t)NUM_SMS * w) * (copy ? 1.f : TILE_UNCACHED_ROW_COST);
+    for (int w = wmax; w >= 1 && w >= wmax / 2; --w) {
+      const long long cost = ceil_div(c, (int64_t)NUM_SMS * w) * w;
       if (warps == 0 || cost < best) {
         best = cost;
         warps = w;
-        in_smem = copy != 0;
       }
     }
   }
   if (warps < 1) return THANOS_ERR_SHAPE;
-  const TileSolveLayout lay = tile_solve_layout(Bw, T, in_smem);
-  const size_t smem = 4 * (size_t)lay.mat_floats + (size_t)warps * lay.per_warp_bytes;
+  const TileSolveLayout lay = tile_solve_layout(Bw, T);
+  const size_t smem = (size_t)warps * lay.per_warp_bytes;
   {
     static std::atomic<unsigned long long> done{0};
     THANOS_CUDA(ensure_max_dyn_smem(solve_rows_tile_kernel, (int)TILE_SMEM_BUDGET, done));
@@ -629,7 +629,7 @@ thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G
   int64_t grid = ceil_div(c, warps);
   if (grid > NUM_SMS) grid = NUM_SMS;
   solve_rows_tile_kernel<<<(unsigned)grid, warps * 32, smem, stream>>>(
-      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, T, in_smem ? 1 : 0, row_lists,
+      Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, T, row_lists,
       list_counts, fixed_kind, report_max_s, stats);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
