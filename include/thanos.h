@@ -100,6 +100,19 @@ thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X,
                                           void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * thanos_hessian_accumulate with a fixed order of floating-point summation (Section 3.2, as
+ * above): a call is not split into concurrent token slices, so every entry of H receives exactly
+ * one addend per call and the result -- hence the factor, the masks and the pruned weights that
+ * follow from it -- is the same bit for bit from run to run for the same sequence of calls.
+ * Same arguments and workspace.  A call with few tokens on a wide layer fills fewer SMs than the
+ * unordered call would (its last wave of tiles can be up to half empty); calls of 16384 tokens
+ * and more lose a few per cent.
+ */
+thanos_status_t thanos_hessian_accumulate_ordered(float* H, int64_t b, const void* X,
+                                                  thanos_dtype_t xdtype, int64_t n_tok, int64_t ldx,
+                                                  void* workspace, size_t ws_bytes, void* stream);
+
+/*
  * Factor the damped Hessian so that the inverse of every trailing block is available
  * (Algorithm 1, last line of the block loop: the Hessian is restricted to the unseen columns
  * and re-inverted for every block; Appendix F.7 counts that as O(b^4 / B)).  This call

@@ -82,6 +82,8 @@ def load_library():
     vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
     lib.thanos_hessian_accumulate.argtypes = [vp, i64, vp, i32, i64, i64, vp, sz, vp]
     lib.thanos_hessian_accumulate.restype = i32
+    lib.thanos_hessian_accumulate_ordered.argtypes = [vp, i64, vp, i32, i64, i64, vp, sz, vp]
+    lib.thanos_hessian_accumulate_ordered.restype = i32
     lib.thanos_prepare_inverse.argtypes = [vp, i64, ctypes.c_float, vp, vp, vp, sz, vp, vp]
     lib.thanos_prepare_inverse.restype = i32
     lib.thanos_prune_layer.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, i32, ctypes.c_double,
@@ -182,10 +184,12 @@ def hessian_status(workspace: torch.Tensor) -> int:
 
 
 def hessian_accumulate(H: torch.Tensor, X: torch.Tensor, stream=None,
-                       workspace: Optional[torch.Tensor] = None, check: bool = False) -> None:
+                       workspace: Optional[torch.Tensor] = None, check: bool = False,
+                       ordered: bool = False) -> None:
     """H += 2 X^T X for tokens-major X [n_tok, b] (float32 or bfloat16); H float32 [b, b].
     With check=True the call's device status word is read back (this waits for the call) and a
-    non-zero status raises."""
+    non-zero status raises.  ordered=True calls thanos_hessian_accumulate_ordered (fixed
+    summation order: bit-reproducible results)."""
     lib = load_library()
     if not X.is_cuda or X.stride(-1) != 1:
         raise ValueError("X must be a CUDA tensor with unit inner stride")
@@ -197,9 +201,9 @@ def hessian_accumulate(H: torch.Tensor, X: torch.Tensor, stream=None,
     if workspace is None:
         workspace = _ws(workspace_bytes(WS_HESSIAN, 0, b, 0, dt), H.device)
     with _on(H):
-        _check(lib.thanos_hessian_accumulate(H.data_ptr(), b, X.data_ptr(), dt, n_tok, ldx,
-                                             workspace.data_ptr(), workspace.numel(),
-                                             _stream_ptr(stream)), "thanos_hessian_accumulate")
+        fn = lib.thanos_hessian_accumulate_ordered if ordered else lib.thanos_hessian_accumulate
+        _check(fn(H.data_ptr(), b, X.data_ptr(), dt, n_tok, ldx, workspace.data_ptr(),
+                  workspace.numel(), _stream_ptr(stream)), "thanos_hessian_accumulate")
         if check and n_tok > 0:
             st = hessian_status(workspace)
             if st != 0:

@@ -6,12 +6,10 @@ namespace thanos {
 
 std::atomic<long long> g_launch_count{0};
 
-thanos_status_t hessian_accumulate_simt(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
-                                        int64_t n_tok, int64_t ldx, cudaStream_t stream);
 size_t hessian_workspace_bytes(int64_t b, thanos_dtype_t dtype);
 thanos_status_t hessian_accumulate_impl(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
                                         int64_t n_tok, int64_t ldx, void* workspace,
-                                        size_t ws_bytes, cudaStream_t stream);
+                                        size_t ws_bytes, cudaStream_t stream, bool ordered);
 size_t prepare_workspace_bytes(int64_t b);
 thanos_status_t prepare_inverse_impl(const float* H, int64_t b, float damp_rel, float* factor,
                                      float* xnorm, void* workspace, size_t ws_bytes,
@@ -112,9 +110,10 @@ using namespace thanos;
 
 extern "C" {
 
-thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
-                                          int64_t n_tok, int64_t ldx, void* workspace,
-                                          size_t ws_bytes, void* stream) {
+static thanos_status_t hessian_accumulate_checked(float* H, int64_t b, const void* X,
+                                                  thanos_dtype_t xdtype, int64_t n_tok, int64_t ldx,
+                                                  void* workspace, size_t ws_bytes, void* stream,
+                                                  bool ordered) {
   if (!H || (!X && n_tok > 0)) return THANOS_ERR_INVALID_ARG;
   if (!dtype_ok(xdtype)) return THANOS_ERR_DTYPE;
   if (b < 8 || b > MAX_B || b % 8 != 0 || n_tok < 0) return THANOS_ERR_SHAPE;
@@ -124,7 +123,19 @@ thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X, th
   if (ws_bytes < hessian_workspace_bytes(b, xdtype) || (!workspace && ws_bytes > 0))
     return THANOS_ERR_WORKSPACE;
   return hessian_accumulate_impl(H, b, X, xdtype, n_tok, ldx, workspace, ws_bytes,
-                                 static_cast<cudaStream_t>(stream));
+                                 static_cast<cudaStream_t>(stream), ordered);
+}
+
+thanos_status_t thanos_hessian_accumulate(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
+                                          int64_t n_tok, int64_t ldx, void* workspace,
+                                          size_t ws_bytes, void* stream) {
+  return hessian_accumulate_checked(H, b, X, xdtype, n_tok, ldx, workspace, ws_bytes, stream, false);
+}
+
+thanos_status_t thanos_hessian_accumulate_ordered(float* H, int64_t b, const void* X,
+                                                  thanos_dtype_t xdtype, int64_t n_tok, int64_t ldx,
+                                                  void* workspace, size_t ws_bytes, void* stream) {
+  return hessian_accumulate_checked(H, b, X, xdtype, n_tok, ldx, workspace, ws_bytes, stream, true);
 }
 
 thanos_status_t thanos_prepare_inverse(const float* H, int64_t b, float damp_rel, float* factor,

@@ -55,15 +55,18 @@ hessian_syrk_simt_kernel(float* __restrict__ H, int b, const T* __restrict__ X, 
 }  // namespace
 
 thanos_status_t hessian_accumulate_simt(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
-                                        int64_t n_tok, int64_t ldx, cudaStream_t stream) {
+                                        int64_t n_tok, int64_t ldx, cudaStream_t stream,
+                                        bool ordered) {
   int nt = (int)ceil_div(b, HB);
   int npairs = nt * (nt + 1) / 2;
   // slice tokens so the grid has a few waves of CTAs; each slice is at most 2^30 tokens
-  int64_t want_slices = ceil_div(NUM_SMS * 4, npairs);
+  // ordered: one slice, so that every entry of H receives exactly one addend per call
+  int64_t want_slices = ordered ? 1 : ceil_div(NUM_SMS * 4, npairs);
   int64_t tok_per_slice = ceil_div(n_tok, want_slices);
   tok_per_slice = round_up((size_t)(tok_per_slice < 256 ? 256 : tok_per_slice), HK);
   if (tok_per_slice > (1 << 30)) tok_per_slice = 1 << 30;
   int64_t slices = ceil_div(n_tok, tok_per_slice);
+  if (ordered && slices != 1) return THANOS_ERR_SHAPE;
   if (slices > 65535) return THANOS_ERR_SHAPE;
   dim3 grid(npairs, (unsigned)slices);
   if (xdtype == THANOS_F32) {

@@ -322,7 +322,7 @@ __global__ void split_planes_kernel(const float* __restrict__ X, int64_t ldx, in
 
 thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld_elems, int n_tok,
                           int planes, int64_t plane_stride_elems, int32_t* status,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, bool one_slice) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return THANOS_ERR_CUDA;
   CUtensorMap tmap;
@@ -362,7 +362,8 @@ thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld
     if (eff_of[s] > best_eff) best_eff = eff_of[s];
   }
   int best_s = 1;
-  while (best_s < max_s && eff_of[best_s] < best_eff - 0.03) ++best_s;
+  // one slice: every entry of H then receives exactly one addend per launch (fixed summation order)
+  while (!one_slice && best_s < max_s && eff_of[best_s] < best_eff - 0.03) ++best_s;
   int st = (n_tok + best_s - 1) / best_s;
   st = (st + FLUSH_STAGES * BK - 1) / (FLUSH_STAGES * BK) * (FLUSH_STAGES * BK);
   p.slice_tokens = st;
@@ -396,7 +397,7 @@ constexpr int SPLIT_CHUNK = 8192;  // tokens of fp32 input split per pass
 
 bool hessian_tc2_supported(int64_t b, int64_t n_tok);
 thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, int64_t ld_elems,
-                                   int n_tok, int32_t* status, cudaStream_t stream);
+                                   int n_tok, int32_t* status, cudaStream_t stream, bool one_slice);
 
 size_t hessian_tc_workspace_bytes(int64_t b, thanos_dtype_t dtype) {
   size_t w = 256;  // status word
@@ -408,7 +409,7 @@ bool hessian_tc_supported(int64_t b, int64_t n_tok) { return b >= 256 && n_tok >
 
 thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos_dtype_t xdtype,
                                       int64_t n_tok, int64_t ldx, void* workspace,
-                                      cudaStream_t stream) {
+                                      cudaStream_t stream, bool ordered) {
   int32_t* status = static_cast<int32_t*>(workspace);
   THANOS_CUDA(cudaMemsetAsync(status, 0, 16, stream));
   if (xdtype == THANOS_BF16) {
@@ -418,12 +419,13 @@ thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos
       int64_t n = n_tok - t0 < step ? n_tok - t0 : step;
       if (hessian_tc2_supported(b, n)) {  // CTA pairs; falls through if they cannot be scheduled
         thanos_status_t st2 = launch_hessian_tc2(
-            H, (int)b, static_cast<const __nv_bfloat16*>(X) + t0 * ldx, ldx, (int)n, status, stream);
+            H, (int)b, static_cast<const __nv_bfloat16*>(X) + t0 * ldx, ldx, (int)n, status, stream,
+            ordered);
         if (st2 == THANOS_OK) continue;
         if (st2 != THANOS_ERR_SHAPE) return st2;
       }
       THANOS_TRY(launch_tc(H, (int)b, static_cast<const __nv_bfloat16*>(X) + t0 * ldx, ldx, (int)n,
-                           1, n * ldx, status, stream));
+                           1, n * ldx, status, stream, ordered));
     }
     return THANOS_OK;
   }
@@ -433,7 +435,7 @@ thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos
     split_planes_kernel<<<NUM_SMS * 8, 256, 0, stream>>>(static_cast<const float*>(X) + t0 * ldx, ldx,
                                                      n, (int)b, planes);
     THANOS_CHECK_LAUNCH();
-    THANOS_TRY(launch_tc(H, (int)b, planes, b, n, 3, (int64_t)n * b, status, stream));
+    THANOS_TRY(launch_tc(H, (int)b, planes, b, n, 3, (int64_t)n * b, status, stream, ordered));
   }
   return THANOS_OK;
 }

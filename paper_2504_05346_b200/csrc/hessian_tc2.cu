@@ -41,6 +41,7 @@ struct Params2 {
   int n_tiles;         // 256-blocks pairs (I <= J)
   int n_slices;
   int slice_tokens;    // multiple of BK
+  int sb;              // super-block edge in tiles
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -116,18 +117,49 @@ struct Unit2 {
   int I, J, t0, nst;
   bool diag;
 };
+// Tiles are numbered super-block by super-block (SB x SB tiles, upper triangle of super-blocks in
+// column order): the pairs that run at the same time then share a handful of feature blocks of
+// the same token slice, which the L2 serves -- in plain column order a wave of tiles spans most
+// row blocks of a wide layer and every wave re-reads most of X from DRAM.
 __device__ __forceinline__ Unit2 decode_unit2(const Params2& p, int u) {
   Unit2 r;
   int tile = u % p.n_tiles;
   const int slice = u / p.n_tiles;
-  int J = 0;
-  while (tile > J) {  // column block J has J + 1 row blocks
-    tile -= J + 1;
-    ++J;
+  const int nT = (p.b + TT - 1) / TT;
+  const int SB = p.sb;
+  const int nS = (nT + SB - 1) / SB;
+  int I = 0, J = 0;
+  for (int SJ = 0; SJ < nS; ++SJ) {
+    const int wj = min(SB, nT - SJ * SB);
+    bool found = false;
+    for (int SI = 0; SI <= SJ; ++SI) {
+      const int wi = min(SB, nT - SI * SB);
+      const int size = SI == SJ ? (wj * (wj + 1)) / 2 : wi * wj;
+      if (tile < size) {
+        int di, dj;
+        if (SI == SJ) {
+          dj = 0;
+          while (tile > dj) {  // column dj of the triangle has dj + 1 tiles
+            tile -= dj + 1;
+            ++dj;
+          }
+          di = tile;
+        } else {
+          di = tile / wj;
+          dj = tile - di * wj;
+        }
+        I = SI * SB + di;
+        J = SJ * SB + dj;
+        found = true;
+        break;
+      }
+      tile -= size;
+    }
+    if (found) break;
   }
-  r.I = tile;
+  r.I = I;
   r.J = J;
-  r.diag = tile == J;
+  r.diag = I == J;
   r.t0 = slice * p.slice_tokens;
   int t1 = r.t0 + p.slice_tokens;
   if (t1 > p.n_tok) t1 = p.n_tok;
@@ -375,7 +407,7 @@ bool hessian_tc2_supported(int64_t b, int64_t n_tok) { return b >= 1024 && n_tok
 // bf16 X [n_tok, b] (leading dimension ld_elems); returns THANOS_ERR_SHAPE when CTA pairs cannot
 // be scheduled on this device (the caller then uses the one-CTA kernel).
 thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, int64_t ld_elems,
-                                   int n_tok, int32_t* status, cudaStream_t stream) {
+                                   int n_tok, int32_t* status, cudaStream_t stream, bool one_slice) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return THANOS_ERR_CUDA;
   {
@@ -400,6 +432,7 @@ thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, i
   p.n_tok = n_tok;
   const int nT = (b + TT - 1) / TT;
   p.n_tiles = nT * (nT + 1) / 2;
+  p.sb = 8;  // 64 tiles per super-block: about one wave of the 74 pairs
   // token slices: the count (each slice >= 2048 tokens) that wastes the least of the last wave
   // fewest slices whose last wave wastes at most 3 percent more than the best count does:
   // longer slices mean fewer write-outs of a tile
@@ -415,7 +448,8 @@ thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, i
     if (eff_of[s] > best_eff) best_eff = eff_of[s];
   }
   int best_s = 1;
-  while (best_s < max_s && eff_of[best_s] < best_eff - 0.03) ++best_s;
+  // one slice: every entry of H then receives exactly one addend per launch (fixed summation order)
+  while (!one_slice && best_s < max_s && eff_of[best_s] < best_eff - 0.03) ++best_s;
   int st = (n_tok + best_s - 1) / best_s;
   st = (st + FLUSH_STAGES * BK - 1) / (FLUSH_STAGES * BK) * (FLUSH_STAGES * BK);
   p.slice_tokens = st;

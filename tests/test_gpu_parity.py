@@ -427,6 +427,31 @@ def test_sweep_is_deterministic(T):
     assert torch.equal(a[0], b_[0]) and torch.equal(a[1], b_[1])
 
 
+@pytest.mark.parametrize("dtype,b,a", [("bf16", 1024, 20000), ("f32", 512, 9000), ("bf16", 2048, 33000)])
+def test_ordered_hessian_makes_the_whole_path_reproducible(T, dtype, b, a):
+    """thanos_hessian_accumulate_ordered at widths where the unordered call splits its tokens into
+    concurrent slices: two runs give the same H bit for bit (and with it the same factor, masks and
+    weights); the ordered H is the unordered one up to rounding."""
+    c = 128
+    W = WL.make_weight(c, b, dtype, seed=57)
+    Xd = _acts(a, b, dtype, seed=10 + b, mix=0.3).to(DEV)
+    runs = []
+    for _ in range(2):
+        H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+        T.hessian_accumulate(H, Xd[:a // 2], ordered=True)
+        T.hessian_accumulate(H, Xd[a // 2:], ordered=True)
+        U, xn = T.prepare_inverse(H, 0.01)
+        Wp, M, st = T.prune_layer(W.to(DEV), U, xn, T.UNSTRUCTURED, p=0.5, B=128)
+        runs.append((H, U, xn, Wp, M))
+    for x, y in zip(*runs):
+        assert torch.equal(x, y)
+    Hu = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(Hu, Xd)
+    assert PU.rel_fro(_np64(runs[0][0]), _np64(Hu)) <= 1e-6
+    assert PU.rel_fro(_np64(Hu), O.hessian(_np64(Xd).T)) <= PU.TOL_H
+    assert PU.rel_fro(_np64(runs[0][0]), O.hessian(_np64(Xd).T)) <= PU.TOL_H
+
+
 def test_argument_errors_are_reported(T):
     b = 64
     H = _equal_norm_hessian(b).to(DEV)
