@@ -748,31 +748,56 @@ def test_opt125m_layer_shapes_full_oracle(T, layer):
     assert out["mismatch"] <= 4
 
 
-@pytest.mark.parametrize("mode", ["nm", "unstructured"])
-def test_llama2_70b_width_8192_sampled_rows(T, mode):
-    """The 8192-wide projection of the LLaMA-2-70B-shaped set (2:4 and 60 % unstructured,
-    B = 128, bf16) with 512 rows: counts, exact zeros, and a float64 replay of sampled rows under
-    the GPU's mask."""
+@pytest.mark.parametrize("mode,c", [("nm", 28672), ("unstructured", 8192)],
+                         ids=["gate_28672x8192_2of4", "q_8192x8192_unstr60"])
+def test_llama2_70b_width_8192_full_shapes(T, mode, c):
+    """The 8192-wide layers of the LLaMA-2-70B-shaped set at their own shapes (28672 x 8192 with
+    2:4, 8192 x 8192 with 60 % unstructured, B = 128, bf16): counts, exact zeros, and a float64
+    replay of sampled rows under the GPU's mask."""
     cfg = WL.CONFIGS["llama2_70b"]
-    c, b, B = 512, 8192, cfg.B
+    b, B = 8192, cfg.B
     W = WL.make_weight(c, b, "bf16", seed=cfg.seed, layer_index=0, device=DEV)
     Xd = WL.config_activations(cfg, 0, b, device=DEV, a=12288)
     H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
     T.hessian_accumulate(H, Xd)
+    del Xd
     U, xn = T.prepare_inverse(H, cfg.damp_rel)
     if mode == "nm":
         Wp, M, st = T.prune_layer(W, U, xn, T.NM, n=2, m=4, B=B)
         assert bool((M.view(c, b // 4, 4).sum(dim=2) == 2).all())
+        assert st.n_pruned == c * b // 2
     else:
         Wp, M, st = T.prune_layer(W, U, xn, T.UNSTRUCTURED, p=0.6, B=B)
         assert st.n_pruned == PU.expected_removed(0.6, c, b) and st.r_left == 0
         assert st.select_misses <= 2
     assert st.n_blocks == b // B and bool((Wp[M.bool()] == 0).all())
     Hd = O.damped(_np64(H), cfg.damp_rel)
-    rows = np.array([0, 255, 511])
-    Wr = O.replay_rows(_np64(W)[rows], M.cpu().numpy()[rows], Hd, B)
+    rows = torch.tensor([0, c // 3, c - 1], device=DEV)
+    Wr = O.replay_rows(_np64(W[rows]), M[rows].cpu().numpy(), Hd, B)
     Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
-    assert PU.rel_fro(_np64(Wp)[rows], Wr) <= PU.TOL_W_BF16
+    assert PU.rel_fro(_np64(Wp[rows]), Wr) <= PU.TOL_W_BF16
+
+
+def test_llama3_8b_gate_projection_full_shape(T):
+    """14336 x 4096 (gate / up of the LLaMA-3-8B-shaped set), 4:8, B = 256, bf16, all rows: the
+    CTA-per-row solve at its real row count; pattern, zeros, sampled float64 replay."""
+    cfg = WL.CONFIGS["llama3_8b"]
+    c, b, B = 14336, 4096, cfg.B
+    W = WL.make_weight(c, b, "bf16", seed=cfg.seed, layer_index=4, device=DEV)
+    Xd = WL.config_activations(cfg, 2, b, device=DEV, a=16384)
+    H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
+    T.hessian_accumulate(H, Xd)
+    del Xd
+    U, xn = T.prepare_inverse(H, cfg.damp_rel)
+    Wp, M, st = T.prune_layer(W, U, xn, T.NM, n=cfg.n, m=cfg.m, B=B)
+    assert bool((M.view(c, b // 8, 8).sum(dim=2) == 4).all())
+    assert st.n_pruned == c * b // 2 and st.n_blocks == b // B and st.max_s == B // 2
+    assert bool((Wp[M.bool()] == 0).all())
+    Hd = O.damped(_np64(H), cfg.damp_rel)
+    rows = torch.tensor([0, 5000, c - 1], device=DEV)
+    Wr = O.replay_rows(_np64(W[rows]), M[rows].cpu().numpy(), Hd, B)
+    Wr = _np64(torch.tensor(Wr).to(torch.bfloat16))
+    assert PU.rel_fro(_np64(Wp[rows]), Wr) <= PU.TOL_W_BF16
 
 
 def test_threshold_jumps_between_blocks(T):
