@@ -206,25 +206,42 @@ __device__ __forceinline__ int factor_diag_tile_inv(float* __restrict__ Tt, floa
 }
 
 // Fragment of L_KK^{-1} (lower triangular) from a factored diagonal tile: entry (i, j), j < i, is
-// stored transposed at (j, i); the diagonal is invd.
-__device__ __forceinline__ void load_inverse_frag(const float* __restrict__ Tt,
-                                                  const float* __restrict__ invd16, int g, int t,
-                                                  PanelFrag& f) {
-  float v[4][2];
+// stored transposed at (j, i); the diagonal is invd.  Where a lane's eight entries sit depends on
+// the lane only: `off` holds the tile offsets of the entries below the diagonal, bit e of `below`
+// / `ondiag` says which kind entry e is (entry 2 w + e: row g + 8 (w & 1), column
+// 2t + 8 (w >> 1) + e).
+struct InvFragOff {
+  int off[8];
+  unsigned below, ondiag;
+};
+__device__ __forceinline__ InvFragOff make_inv_frag_off(int g, int t) {
+  InvFragOff f;
+  f.below = f.ondiag = 0;
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
     const int row = g + 8 * (w & 1);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int col = 2 * t + 8 * (w >> 1) + e;
-      float x = 0.f;
-      if (col < row) x = Tt[elem_off(col, row)];
-      else if (col == row) x = invd16[row];
-      v[w][e] = x;
+      f.off[2 * w + e] = col < row ? elem_off(col, row) : 0;
+      if (col < row) f.below |= 1u << (2 * w + e);
+      if (col == row) f.ondiag |= 1u << (2 * w + e);
     }
   }
+  return f;
+}
+__device__ __forceinline__ void load_inverse_frag(const float* __restrict__ Tt,
+                                                  const float* __restrict__ invd16, int g,
+                                                  const InvFragOff& io, PanelFrag& f) {
+  const float d0 = invd16[g], d1 = invd16[g + 8];
+  float v[8];
 #pragma unroll
-  for (int w = 0; w < 4; ++w) split_pair(v[w][0], v[w][1], f.w[0][w], f.w[1][w], f.w[2][w]);
+  for (int i = 0; i < 8; ++i) {
+    const float x = Tt[io.off[i]];  // offset 0 (a valid entry) where the value is not used
+    v[i] = (io.below >> i) & 1u ? x : ((io.ondiag >> i) & 1u ? ((i >> 1) & 1 ? d1 : d0) : 0.f);
+  }
+#pragma unroll
+  for (int w = 0; w < 4; ++w) split_pair(v[2 * w], v[2 * w + 1], f.w[0][w], f.w[1][w], f.w[2][w]);
 }
 
 // One warp per row; the arguments and the split of the CTAs between the two kinds of rows are
@@ -252,6 +269,12 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   unsigned short* klist = qlist + Bw + 16;
   const int g = lane >> 2, t4 = lane & 3;
   const FragOff fo = make_frag_off(g, t4);
+  const InvFragOff io = make_inv_frag_off(g, t4);
+  // forward substitution: lane (l = lane % 16, half = lane / 16) reads column l of the upper
+  // triangle of a diagonal tile, rows 8 half .. 8 half + 7
+  int fwd_off[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) fwd_off[e] = elem_off(8 * (lane >> 4) + e, lane & 15);
   // gather: lane (r0 = lane / 16, k = lane % 16) fills rows r0 + 2 h of column k of a tile
   int gofs[8];
 #pragma unroll
@@ -429,7 +452,7 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         if (m == 0) break;
         // panel tiles as products with the inverse of the diagonal factor
         PanelFrag fl, f0, f1, f2;
-        load_inverse_frag(Lk, invd + 16 * K, g, t4, fl);
+        load_inverse_frag(Lk, invd + 16 * K, g, io, fl);
         {
           PanelFrag fa;
           load_panel_frag(A + tbase(K + 1, K), fo, fa);
@@ -505,11 +528,12 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         const float4 v1 = *reinterpret_cast<const float4*>(yv + 16 * I + 8 * hh + 4);
         const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
         float acc = 0.f;
+        const float dl = invd[16 * I + l16];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const int cidx = 8 * hh + e;
-          const float x = cidx < l16 ? Lk[elem_off(cidx, l16)] : (cidx == l16 ? invd[16 * I + l16] : 0.f);
-          acc = fmaf(x, vv[e], acc);
+          const float x = Lk[fwd_off[e]];  // entries on or below the diagonal are not used
+          acc = fmaf(cidx < l16 ? x : (cidx == l16 ? dl : 0.f), vv[e], acc);
         }
         acc += __shfl_xor_sync(FULL, acc, 16);
         __syncwarp();
