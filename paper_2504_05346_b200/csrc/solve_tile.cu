@@ -155,36 +155,32 @@ __device__ __forceinline__ void panel_product(float* __restrict__ Tt, const Pane
 // [L; L^{-T}].  Every lane also carries its own diagonal entry, so the pivot of the next column
 // does not wait for the updates of the others.  Stored: L in the lower triangle and diagonal of
 // the tile, the strict upper triangle of L^{-T} above it, 1 / l_jj (the diagonal of L^{-1}) in
-// invd.  Columns col0 + j >= n (identity padding) get pivot 1.  Returns the first column with a
-// pivot that is not positive, -1 if there is none.
-__device__ __forceinline__ int factor_diag_tile_inv(float* __restrict__ Tt, float* __restrict__ invd,
-                                                    int col0, int n, int lane) {
+// invd.  Columns col0 + j >= n (identity padding) get pivot 1.  Returns whether a pivot was not
+// positive and finite.  `ident` is an identity tile in the tile layout, rc / doff the offsets of
+// the chunks and of the diagonal entry of row lane % 16.
+__device__ __forceinline__ bool factor_diag_tile_inv(float* __restrict__ Tt,
+                                                     const float* __restrict__ ident,
+                                                     float* __restrict__ invd, int col0, int n,
+                                                     int lane, const int (&rc)[4], int doff) {
   const int r = lane & 15;
   const bool top = lane < 16;
+  // rows of the tile for lanes 0..15, rows of the identity (same tile layout) for lanes 16..31
+  const float* src = top ? Tt : ident;
   float a[16];
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    const float4 v = *reinterpret_cast<const float4*>(Tt + chunk_off(r, c));
+    const float4 v = *reinterpret_cast<const float4*>(src + rc[c]);
     a[4 * c] = v.x; a[4 * c + 1] = v.y; a[4 * c + 2] = v.z; a[4 * c + 3] = v.w;
   }
-  float diag = 0.f;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    if (r == j) diag = a[j];
-    if (!top) a[j] = (r == j) ? 1.f : 0.f;
-  }
-  int bad = -1;
+  float diag = Tt[doff];
+  const int nlive = n - col0;  // columns beyond it are identity padding
+  bool bad = false;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     float dj = __shfl_sync(FULL, diag, j);
-    if (col0 + j < n) {
-      if (!(dj > 0.f) || !isfinite(dj)) {
-        if (bad < 0) bad = col0 + j;
-        dj = 1.f;
-      }
-    } else {
-      dj = 1.f;
-    }
+    const bool okp = dj > 0.f && dj < 3.0e38f;  // positive and finite
+    if (j < nlive && !okp) bad = true;
+    dj = (j < nlive && okp) ? dj : 1.f;
     const float rinv = rsqrtf(dj);
     if (lane == 0) invd[col0 + j] = rinv;
     a[j] *= rinv;
@@ -199,7 +195,7 @@ __device__ __forceinline__ int factor_diag_tile_inv(float* __restrict__ Tt, floa
   // half-warp (L^{-T})
 #pragma unroll
   for (int cidx = 0; cidx < 16; ++cidx) {
-    if (top ? (cidx <= r) : (cidx > r)) Tt[elem_off(r, cidx)] = a[cidx];
+    if (top ? (cidx <= r) : (cidx > r)) Tt[rc[cidx >> 2] + (cidx & 3)] = a[cidx];
   }
   __syncwarp();
   return bad;
@@ -270,6 +266,15 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   const int g = lane >> 2, t4 = lane & 3;
   const FragOff fo = make_frag_off(g, t4);
   const InvFragOff io = make_inv_frag_off(g, t4);
+  // chunk offsets and diagonal entry of tile row lane % 16
+  int rc[4];
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) rc[cc] = chunk_off(lane & 15, cc);
+  const int doff = elem_off(lane & 15, lane & 15);
+  // an identity tile (the lower half-warp of a diagonal factorisation starts from its rows)
+  __shared__ __align__(16) float s_ident[256];
+  for (int e = threadIdx.x; e < 256; e += blockDim.x) s_ident[elem_off(e >> 4, e & 15)] = (e >> 4) == (e & 15) ? 1.f : 0.f;
+  __syncthreads();
   // forward substitution: lane (l = lane % 16, half = lane / 16) reads column l of the upper
   // triangle of a diagonal tile, rows 8 half .. 8 half + 7
   int fwd_off[8];
@@ -447,7 +452,7 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       bool bad = false;
       for (int K = 0; K < T; ++K) {
         float* Lk = A + tbase(K, K);
-        bad |= factor_diag_tile_inv(Lk, invd, 16 * K, n, lane) >= 0;
+        bad |= factor_diag_tile_inv(Lk, s_ident, invd, 16 * K, n, lane, rc, doff);
         const int m = T - K - 1;  // tile rows below the diagonal tile (warp-uniform, <= 3)
         if (m == 0) break;
         // panel tiles as products with the inverse of the diagonal factor
@@ -508,8 +513,8 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           float acc = 0.f;
           for (int J = 0; J < I; ++J) {
             const float* Lt = A + tbase(I, J);
-            const float4 a0 = *reinterpret_cast<const float4*>(Lt + chunk_off(l16, 2 * hh));
-            const float4 a1 = *reinterpret_cast<const float4*>(Lt + chunk_off(l16, 2 * hh + 1));
+            const float4 a0 = *reinterpret_cast<const float4*>(Lt + (hh ? rc[2] : rc[0]));
+            const float4 a1 = *reinterpret_cast<const float4*>(Lt + (hh ? rc[3] : rc[1]));
             const float4 y0 = *reinterpret_cast<const float4*>(yv + 16 * J + 8 * hh);
             const float4 y1 = *reinterpret_cast<const float4*>(yv + 16 * J + 8 * hh + 4);
             acc = fmaf(a0.x, y0.x, acc); acc = fmaf(a0.y, y0.y, acc);
@@ -546,8 +551,8 @@ solve_rows_tile_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         const float* Lk = A + tbase(Kb, Kb);
         {
           // row l of L^{-T}: columns > l in the tile's upper triangle, the diagonal in invd
-          const float4 a0 = *reinterpret_cast<const float4*>(Lk + chunk_off(l16, 2 * hh));
-          const float4 a1 = *reinterpret_cast<const float4*>(Lk + chunk_off(l16, 2 * hh + 1));
+          const float4 a0 = *reinterpret_cast<const float4*>(Lk + (hh ? rc[2] : rc[0]));
+          const float4 a1 = *reinterpret_cast<const float4*>(Lk + (hh ? rc[3] : rc[1]));
           const float4 v0 = *reinterpret_cast<const float4*>(yv + 16 * Kb + 8 * hh);
           const float4 v1 = *reinterpret_cast<const float4*>(yv + 16 * Kb + 8 * hh + 4);
           const float aa[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
@@ -633,7 +638,7 @@ thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G
   long long best = 0;
   {
     const TileSolveLayout l = tile_solve_layout(Bw, T);
-    int wmax = (int)(TILE_SMEM_BUDGET / l.per_warp_bytes);
+    int wmax = (int)((TILE_SMEM_BUDGET - 1024 /* static identity tile */) / l.per_warp_bytes);
     if (wmax > TILE_MAX_WARPS) wmax = TILE_MAX_WARPS;
     for (int w = wmax; w >= 1 && w >= wmax / 2; --w) {
       const long long cost = ceil_div(c, (int64_t)NUM_SMS * w) * w;
@@ -648,7 +653,7 @@ thanos_status_t launch_tile_solve(float* Wc, const uint8_t* mask, const float* G
   const size_t smem = (size_t)warps * lay.per_warp_bytes;
   {
     static std::atomic<unsigned long long> done{0};
-    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_tile_kernel, (int)TILE_SMEM_BUDGET, done));
+    THANOS_CUDA(ensure_max_dyn_smem(solve_rows_tile_kernel, (int)TILE_SMEM_BUDGET - 1024, done));
   }
   int64_t grid = ceil_div(c, warps);
   if (grid > NUM_SMS) grid = NUM_SMS;
