@@ -913,9 +913,7 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    // the tie kernels almost always return at once (they work only when a threshold value is
-    // shared by entries on both sides of the cut): a small grid keeps the empty launch short
-    int hg = c < NUM_SMS * 2 ? c : NUM_SMS * 2;
+    int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
     for (int pass = 0; pass < 5; ++pass) {
