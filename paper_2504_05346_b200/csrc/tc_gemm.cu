@@ -288,8 +288,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       const Tile tl = decode_tile(p, t);
       if (tl.skip) continue;
       const int row = tl.m0 + r_in_tile;
-      __nv_bfloat16* prow =
-          p.Dp ? p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)row * p.ldp : nullptr;
       ok = ok && mbar_wait(tfull_bar(q), tphase, abort_flag);
       tc_fence_after();
       {
@@ -306,7 +304,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             for (int j = 0; j < 32; ++j) v[j] = 0u;
           }
           const int cbase = tl.n0 + 64 * h + 32 * cc;
-          if (p.D) {
+          if (p.D || p.Dp) {
             // the buffer is free once TMA has read the previous chunk out of it
             if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             named_bar_sync(1 + 2 * h, 128);
@@ -321,19 +319,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             named_bar_sync(2 + 2 * h, 128);
-            if (issuer && ok && cbase < p.N) {
+            if (issuer && ok && cbase < p.N && p.D) {
               if (p.accumulate) tma_reduce_add_3d(&mapD, stg_addr, cbase, tl.m0, tl.z);
               else tma_store_3d(&mapD, stg_addr, cbase, tl.m0, tl.z);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
           }
-          if (prow && ok && row < p.M) {
+          if (p.Dp && ok) {
+            // Planes of the result from the staging buffer: every warp instruction covers four
+            // rows of 32 columns (64 contiguous bytes per row and plane) instead of one 8-byte
+            // piece in each of 32 rows.  The buffer is not reused before the next chunk's barrier.
+            const int tih = 32 * g + lane;
+            const int c4 = tih & 7;
+            const int col = cbase + 4 * c4;
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const int col = cbase + j;
-              float o[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) o[e] = p.alpha * __uint_as_float(v[j + e]);
+            for (int it = 0; it < 8; ++it) {
+              const int rr = (tih >> 3) + 16 * it;
+              const int grow = tl.m0 + rr;
+              if (grow >= p.M || col >= p.N) continue;
+              const float4 sv =
+                  *reinterpret_cast<const float4*>(stg + rr * 128 + ((c4 ^ (rr & 7)) << 4));
+              float o[4] = {sv.x, sv.y, sv.z, sv.w};
+              __nv_bfloat16* pr = p.Dp + (int64_t)tl.z * p.dp_batch + (int64_t)grow * p.ldp;
               if (col + 3 < p.N) {
 #pragma unroll
                 for (int pl = 0; pl < 3; ++pl) {
@@ -348,14 +355,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                          ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
                   pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) |
                          ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
-                  *reinterpret_cast<uint2*>(prow + (int64_t)pl * p.dp_plane + col) = pk;
+                  *reinterpret_cast<uint2*>(pr + (int64_t)pl * p.dp_plane + col) = pk;
                 }
               } else {
                 for (int e = 0; e < 4 && col + e < p.N; ++e) {
                   float val = o[e];
                   for (int pl = 0; pl < 3; ++pl) {
                     const __nv_bfloat16 hb = __float2bfloat16_rn(val);
-                    prow[(int64_t)pl * p.dp_plane + col + e] = hb;
+                    pr[(int64_t)pl * p.dp_plane + col + e] = hb;
                     val -= __bfloat162float(hb);
                   }
                 }
