@@ -71,14 +71,21 @@ def test_noalloc_calls_leave_device_memory_untouched(T):
                        torch.cuda.current_stream().cuda_stream)
     warm = torch.zeros(64, dtype=torch.uint8, device=DEV)
     assert lib.thanos_prune_layer_noalloc(*args(warm)) == 0      # first call: address look-up
+    import gc
+    gc.collect()   # leftovers of earlier tests must not be freed between the two readings
     torch.cuda.synchronize()
     alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
     free0, _ = torch.cuda.mem_get_info()
-    for st in stats:
-        assert lib.thanos_prune_layer_noalloc(*args(st)) == 0
-    torch.cuda.synchronize()
-    free1, _ = torch.cuda.mem_get_info()
-    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    gc.disable()
+    try:
+        for st in stats:
+            assert lib.thanos_prune_layer_noalloc(*args(st)) == 0
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        alloc1, reserved1 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    finally:
+        gc.enable()
+    assert alloc1 == alloc0 and reserved1 == reserved0
     assert free1 == free0
     assert torch.equal(stats[0], stats[1]) and torch.equal(stats[1], stats[2])
     ref = T.prune_layer(W, U, xn, T.UNSTRUCTURED, p=0.5, B=64)
