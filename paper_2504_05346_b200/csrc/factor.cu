@@ -172,7 +172,7 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
     __syncthreads();
   }
   if (warp == 0 && lane == 0 && bad >= 0) report_error(status, THANOS_ERR_NOT_SPD, k0 + n - 1 - bad);
-  // V22[i][j] = L[n-1-i][n-1-j];  U22[i][j] = inv(L)[n-1-i][n-1-j] = identity row (n-1-j), column n-1-i
+  // U22[i][j] = inv(L)[n-1-i][n-1-j] = identity row (n-1-j), column n-1-i
   for (int i = warp; i < n; i += DIAG_THREADS / 32) {
     for (int c4 = lane * 4; c4 < n; c4 += 128) {
       float u4[4];
@@ -182,8 +182,8 @@ diag_block_kernel(float* __restrict__ V, float* __restrict__ U, __nv_bfloat16* _
         const int j = c4 + e;
         float u = 0.f;
         if (j >= i) {
+          // (the factor V22 itself is not written back: nothing reads this block of V again)
           const int li = n - 1 - i, lj = n - 1 - j;  // lj <= li
-          V[o + e] = tile_at(li >> 4, lj >> 4)[tile::elem_off(li & 15, lj & 15)];
           u = tile_at(Tn + (lj >> 4), li >> 4)[tile::elem_off(lj & 15, li & 15)];
         }
         u4[e] = u;
