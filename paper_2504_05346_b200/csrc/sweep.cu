@@ -913,7 +913,12 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
+    // The tie kernels work only when a threshold value is shared by entries on both sides of the
+    // cut.  Weights that come straight from a 16-bit format do that in the first block; after it
+    // every residual weight has received an fp32 update and the kernels return at once, which a
+    // small grid does faster.
+    const int tie_ctas = j1 == 0 ? NUM_SMS * 8 : NUM_SMS * 2;
+    int hg = c < tie_ctas ? c : tie_ctas;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
     for (int pass = 0; pass < 5; ++pass) {
