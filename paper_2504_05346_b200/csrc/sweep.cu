@@ -913,12 +913,10 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    // The tie kernels work only when a threshold value is shared by entries on both sides of the
-    // cut.  Weights that come straight from a 16-bit format do that in the first block; after it
-    // every residual weight has received an fp32 update and the kernels return at once, which a
-    // small grid does faster.
-    const int tie_ctas = j1 == 0 ? NUM_SMS * 8 : NUM_SMS * 2;
-    int hg = c < tie_ctas ? c : tie_ctas;
+    // The tie kernels work whenever the threshold value is shared by entries on both sides of
+    // the cut -- with tens of millions of fp32 scores in the residual of a wide layer that is
+    // about every second block, not a rare case: they get a full grid.
+    int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
     for (int pass = 0; pass < 5; ++pass) {
