@@ -289,6 +289,7 @@ __device__ __forceinline__ void find_rank_bin(const unsigned* hist, int nbin, un
 // Shared histogram: radix passes keep one counter per (bin, lane) -- a warp never hits the same
 // bank twice, whatever the skew of the metric; bracket / refine passes see few keys inside
 // their range and use plain counters.
+template <int BR_UNROLL>
 __global__ void __launch_bounds__(256)
 select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                    int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
@@ -361,10 +362,21 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
     const int WINDOW_SHIFT = wlog - WINDOW_BINS_LOG2;
     for (int row = blockIdx.x; row < c; row += gridDim.x) {
       const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-#pragma unroll 2
-      for (int q = threadIdx.x; q < w4; q += 256) {
-        const float4 w = wr[q];
-        const float4 x = __ldg(&xr[q]);
+      // BR_UNROLL float4 loads in flight per thread: two when the working copy sits in L2, four
+      // when the residual streams from HBM
+      for (int q0 = threadIdx.x; q0 < w4; q0 += 256 * BR_UNROLL) {
+        float4 wv[BR_UNROLL], xv[BR_UNROLL];
+#pragma unroll
+        for (int u = 0; u < BR_UNROLL; ++u) {
+          const int q = q0 + 256 * u;
+          wv[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          xv[u] = q < w4 ? __ldg(&xr[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < BR_UNROLL; ++u) {
+        if (q0 + 256 * u >= w4) break;
+        const float4 w = wv[u];
+        const float4 x = xv[u];
         const unsigned k0 = metric_key(w.x, x.x), k1 = metric_key(w.y, x.y);
         const unsigned k2 = metric_key(w.z, x.z), k3 = metric_key(w.w, x.w);
         below += (k0 < lo) + (k1 < lo) + (k2 < lo) + (k3 < lo);
@@ -381,6 +393,7 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
               if (pos < (unsigned)CTA_CAND) s_cand[pos] = kk[e];
             }
           }
+        }
         }
       }
     }
@@ -922,9 +935,15 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     for (int pass = 0; pass < 5; ++pass) {
       // passes after the first usually look at the copied keys only, or do nothing
       const int sgp = pass == 0 ? sg : (sg < NUM_SMS * 2 ? sg : NUM_SMS * 2);
-      select_pass_kernel<<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
-                                                 w.list_counts, pass == 0 ? 1 : 0, stats, w.cand,
-                                                 (unsigned)w.cand_cap);
+      // residuals beyond the L2 stream from HBM and want more loads in flight
+      if ((size_t)c * (size_t)(b - j1) * sizeof(float) > ((size_t)96 << 20))
+        select_pass_kernel<4><<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                      w.list_counts, pass == 0 ? 1 : 0, stats,
+                                                      w.cand, (unsigned)w.cand_cap);
+      else
+        select_pass_kernel<2><<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                      w.list_counts, pass == 0 ? 1 : 0, stats,
+                                                      w.cand, (unsigned)w.cand_cap);
       THANOS_CHECK_LAUNCH();
     }
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
