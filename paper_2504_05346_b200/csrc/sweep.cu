@@ -547,6 +547,7 @@ tie_count_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, 
     const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
     const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
     unsigned cnt = 0;
+#pragma unroll 4
     for (int q = threadIdx.x; q < w4; q += 256) {
       float4 w = wr[q];
       float4 x = __ldg(&xr[q]);
