@@ -12,6 +12,8 @@
 //   W[:, j2:] += delta P2      (because -lambda-hat R = delta inv(G) (U_bb^T U[j1:j2, j1:])).
 // G, S, V_bb and P2 depend only on U, so they are computed for all blocks at the start of the
 // sweep.
+#include <cooperative_groups.h>
+
 #include "simt_gemm.cuh"
 #include "tc_gemm.cuh"
 
@@ -290,17 +292,19 @@ __device__ __forceinline__ void find_rank_bin(const unsigned* hist, int nbin, un
 // bank twice, whatever the skew of the metric; bracket / refine passes see few keys inside
 // their range and use plain counters.
 template <int BR_UNROLL>
-__global__ void __launch_bounds__(256)
-select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
-                   int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
-                   unsigned* __restrict__ list_counts, int first_launch, thanos_stats_t* stats,
-                   unsigned* __restrict__ cand, unsigned cand_cap) {
+__device__ __forceinline__ void select_pass_body(const float* __restrict__ Wc,
+                                                 const float* __restrict__ xnorm, int c, int b, int j1,
+                                                 SweepState* st, unsigned* __restrict__ hist,
+                                                 const int64_t* r_ext,
+                                                 unsigned* __restrict__ list_counts, int first_launch,
+                                                 thanos_stats_t* stats, unsigned* __restrict__ cand,
+                                                 unsigned cand_cap) {
   __shared__ unsigned sh[RADIX_BINS * RADIX_REPL];
   __shared__ unsigned s_cand[CTA_CAND];
   __shared__ unsigned s_ncand, s_cbase;
   __shared__ int s_last;
   __shared__ unsigned s_below;
-  const int phase = st->phase;
+  const int phase = *reinterpret_cast<volatile int*>(&st->phase);
   if (phase == PH_DONE && !first_launch) return;
   if (first_launch && blockIdx.x == 0 && threadIdx.x == 0) {
     list_counts[0] = list_counts[1] = 0;
@@ -531,6 +535,36 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
       st->cand_total = 0;
       st->cand_overflow = 0;
     }
+  }
+}
+
+template <int BR_UNROLL>
+__global__ void __launch_bounds__(256)
+select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
+                   int j1, SweepState* st, unsigned* __restrict__ hist, const int64_t* r_ext,
+                   unsigned* __restrict__ list_counts, int first_launch, thanos_stats_t* stats,
+                   unsigned* __restrict__ cand, unsigned cand_cap) {
+  select_pass_body<BR_UNROLL>(Wc, xnorm, c, b, j1, st, hist, r_ext, list_counts, first_launch, stats,
+                              cand, cand_cap);
+}
+
+// The passes a block may still need after its first two launches (bracket + refine, or the first
+// two radix passes): up to three more radix passes, in ONE cooperative launch with a grid barrier
+// between them.  It returns at once when the threshold is known, which is the usual case, so a
+// block step carries one launch that does nothing instead of three.
+template <int BR_UNROLL>
+__global__ void __launch_bounds__(256)
+select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
+                   int j1, SweepState* st, unsigned* __restrict__ hist,
+                   unsigned* __restrict__ list_counts, thanos_stats_t* stats,
+                   unsigned* __restrict__ cand, unsigned cand_cap) {
+  cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+  for (int it = 0; it < 3; ++it) {
+    // the phase only changes between two grid barriers, so every CTA reads the same value
+    if (*reinterpret_cast<volatile int*>(&st->phase) == PH_DONE) return;
+    select_pass_body<BR_UNROLL>(Wc, xnorm, c, b, j1, st, hist, nullptr, list_counts, 0, stats, cand,
+                                cand_cap);
+    grid.sync();
   }
 }
 
@@ -933,11 +967,13 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
-    for (int pass = 0; pass < 5; ++pass) {
-      // passes after the first usually look at the copied keys only, or do nothing
-      const int sgp = pass == 0 ? sg : (sg < NUM_SMS * 2 ? sg : NUM_SMS * 2);
-      // residuals beyond the L2 stream from HBM and want more loads in flight
-      if ((size_t)c * (size_t)(b - j1) * sizeof(float) > ((size_t)96 << 20))
+    // residuals beyond the L2 stream from HBM and want more loads in flight
+    const bool big = (size_t)c * (size_t)(b - j1) * sizeof(float) > ((size_t)96 << 20);
+    const int sg2 = sg < NUM_SMS * 2 ? sg : NUM_SMS * 2;
+    for (int pass = 0; pass < 2; ++pass) {
+      // the second pass usually looks at the copied keys only
+      const int sgp = pass == 0 ? sg : sg2;
+      if (big)
         select_pass_kernel<4><<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
                                                       w.list_counts, pass == 0 ? 1 : 0, stats,
                                                       w.cand, (unsigned)w.cand_cap);
@@ -946,6 +982,25 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
                                                       w.list_counts, pass == 0 ? 1 : 0, stats,
                                                       w.cand, (unsigned)w.cand_cap);
       THANOS_CHECK_LAUNCH();
+    }
+    {
+      // whatever is left of a radix route, behind grid barriers (sg2 <= 2 CTAs per SM: co-resident)
+      const float* a_Wc = Wc;
+      const float* a_xn = xnorm;
+      int a_c = c, a_b = b, a_j1 = j1;
+      SweepState* a_st = w.st;
+      unsigned* a_hist = w.hist;
+      unsigned* a_lc = w.list_counts;
+      thanos_stats_t* a_stats = stats;
+      unsigned* a_cand = w.cand;
+      unsigned a_cap = (unsigned)w.cand_cap;
+      void* args[] = {&a_Wc, &a_xn, &a_c, &a_b, &a_j1, &a_st, &a_hist, &a_lc, &a_stats, &a_cand, &a_cap};
+      const void* fn = big ? reinterpret_cast<const void*>(&select_rest_kernel<4>)
+                           : reinterpret_cast<const void*>(&select_rest_kernel<2>);
+      if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)sg2), dim3(256), args, 0, stream) !=
+          cudaSuccess)
+        return THANOS_ERR_CUDA;
+      count_launch();
     }
     tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
     THANOS_CHECK_LAUNCH();
