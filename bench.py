@@ -275,7 +275,7 @@ def roofline_by_kernel(trace_factor, trace_sweep, cfg, peaks, fp32_peak, masks, 
             upd_elems += float(L.c) * (L.b - j2)
     hbm = peaks["hbm_gbs"]
     if unstructured:
-        ms, n = t_of(trace_sweep, "select_pass_kernel")
+        ms, n = t_of(trace_sweep, "::select_")   # select_pass_kernel and select_rest_kernel
         if ms:
             ach = 4.0 * resid_elems / (ms * 1e-3) / 1e9
             out["select_pass_kernel"] = {

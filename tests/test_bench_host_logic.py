@@ -29,7 +29,8 @@ def test_roofline_by_kernel_from_a_time_table():
     cfg = WL.CONFIGS["tiny"]  # one 256 x 256 layer, B = 64, unstructured
     peaks = {"hbm_gbs": 1000.0, "bf16_tflops": 100.0, "bf16_tflops_sustained": 80.0}
     tr_f = {"thanos::(anonymous namespace)::tc_gemm_kernel(...)": [3, 2.0]}
-    tr_s = {"void thanos::(anonymous namespace)::select_pass_kernel<2>(...)": [20, 1.0],
+    tr_s = {"void thanos::(anonymous namespace)::select_pass_kernel<2>(...)": [20, 0.75],
+            "void thanos::(anonymous namespace)::select_rest_kernel<2>(...)": [4, 0.25],
             "thanos::(anonymous namespace)::tc_gemm_kernel(...)": [3, 0.5],
             "thanos::(anonymous namespace)::solve_rows_tile_kernel(...)": [4, 0.25]}
     M = torch.zeros((256, 256), dtype=torch.uint8)
