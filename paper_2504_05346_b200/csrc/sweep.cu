@@ -637,12 +637,17 @@ tie_scan_kernel(int c, const SweepState* __restrict__ st, const unsigned* __rest
 
 // One warp per row: set the block's mask bytes.  key < tau -> removed; key == tau -> removed
 // while the (row, column)-ordered rank of the tie is below need_eq.
-__global__ void __launch_bounds__(256)
+constexpr int MARK_WARPS = 32;  // rows per CTA and round of the mask kernel
+__global__ void __launch_bounds__(32 * MARK_WARPS)
 mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
                   uint8_t* __restrict__ mask, int c, int b, int j1, int Bw, SweepState* st,
                   const unsigned long long* __restrict__ rowbase, int* __restrict__ row_lists,
                   unsigned* __restrict__ list_counts, thanos_stats_t* stats, int64_t* r_ext) {
   __shared__ int s_last;
+  // the rows of one round of the CTA (one per warp) by kind: the two row lists grow by one
+  // atomic per kind and round instead of one per row
+  __shared__ int s_rows[2][MARK_WARPS];
+  __shared__ unsigned s_cnt[2], s_base[2];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const bool none = st->none != 0;
@@ -651,37 +656,90 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
   const unsigned long long need = st->need_eq;
   unsigned long long total = 0;
   int smax = 0;
-  for (int row = blockIdx.x * 8 + warp; row < c; row += gridDim.x * 8) {
+  for (int row0 = blockIdx.x * MARK_WARPS; row0 < c; row0 += gridDim.x * MARK_WARPS) {
+    const int row = row0 + warp;
+    if (threadIdx.x < 2) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    if (row < c) {
     unsigned long long rank = (none || all_ties) ? 0ull : rowbase[row];
     int s = 0;
-    for (int base = 0; base < Bw; base += 32) {
-      int jj = base + lane;
-      bool in = jj < Bw;
-      unsigned key = 0xffffffffu;
-      if (in) key = metric_key(Wc[(int64_t)row * b + j1 + jj], __ldg(&xnorm[j1 + jj]));
-      bool tie = in && !none && key == tau;
-      unsigned tb = __ballot_sync(0xffffffffu, tie);
-      bool pr = in && !none && key < tau;
-      if (tie) {
-        unsigned long long myrank = rank + __popc(tb & ((1u << lane) - 1u));
-        pr = all_ties || myrank < need;
+    // a lane takes four consecutive columns (Bw % 8 == 0): one 16-byte load of the weights, one of
+    // the norms and one 4-byte store of mask bytes per 128 columns
+    for (int base = 0; base < Bw; base += 128) {
+      const int jj = base + 4 * lane;
+      const bool in = jj < Bw;
+      float4 wv = make_float4(0.f, 0.f, 0.f, 0.f), xv = wv;
+      if (in) {
+        wv = *reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1 + jj);
+        xv = __ldg(reinterpret_cast<const float4*>(xnorm + j1 + jj));
       }
-      rank += __popc(tb);
-      if (in) mask[(int64_t)row * b + j1 + jj] = pr ? 1 : 0;
-      s += __popc(__ballot_sync(0xffffffffu, pr));
+      const unsigned key[4] = {metric_key(wv.x, xv.x), metric_key(wv.y, xv.y),
+                               metric_key(wv.z, xv.z), metric_key(wv.w, xv.w)};
+      bool pr[4];
+      int ntie = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        pr[e] = in && !none && key[e] < tau;
+        ntie += (in && !none && key[e] == tau) ? 1 : 0;
+      }
+      if (__any_sync(0xffffffffu, ntie > 0)) {  // warp-uniform; rare outside tie-heavy blocks
+        // ties in (row, column) order: ties of lower lanes come first, then this lane's in order
+        int incl = ntie;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        unsigned long long myrank = rank + (unsigned long long)(incl - ntie);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (in && !none && key[e] == tau) {
+            pr[e] = all_ties || myrank < need;
+            ++myrank;
+          }
+        }
+        rank += (unsigned long long)__shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (in) {
+        uchar4 mb;
+        mb.x = pr[0] ? 1 : 0;
+        mb.y = pr[1] ? 1 : 0;
+        mb.z = pr[2] ? 1 : 0;
+        mb.w = pr[3] ? 1 : 0;
+        *reinterpret_cast<uchar4*>(mask + (int64_t)row * b + j1 + jj) = mb;
+      }
+      int cnt = (int)pr[0] + (int)pr[1] + (int)pr[2] + (int)pr[3];
+      for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+      s += cnt;
     }
     total += s;
     smax = s > smax ? s : smax;
     if (lane == 0) {
       // rows that remove more than half of the block are solved in the complement form
       const int kind = (s > Bw - s) ? 1 : 0;
-      const unsigned pos = atomicAdd(&list_counts[kind], 1u);
-      row_lists[(size_t)kind * c + pos] = row;
+      s_rows[kind][atomicAdd(&s_cnt[kind], 1u)] = row;
     }
+    }
+    __syncthreads();
+    if (threadIdx.x < 2 && s_cnt[threadIdx.x])
+      s_base[threadIdx.x] = atomicAdd(&list_counts[threadIdx.x], s_cnt[threadIdx.x]);
+    __syncthreads();
+    if (threadIdx.x < MARK_WARPS) {
+      if (threadIdx.x < s_cnt[0]) row_lists[s_base[0] + threadIdx.x] = s_rows[0][threadIdx.x];
+      if (threadIdx.x < s_cnt[1]) row_lists[(size_t)c + s_base[1] + threadIdx.x] = s_rows[1][threadIdx.x];
+    }
+    __syncthreads();
   }
+  // one update of the block's count and of the largest system per CTA
+  if (threadIdx.x < 2) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
   if (lane == 0) {
-    if (total) atomicAdd(&st->blk_count, total);
-    if (smax) atomicMax(&stats->max_s, smax);
+    if (total) atomicAdd(&s_cnt[0], (unsigned)total);
+    if (smax) atomicMax(&s_cnt[1], (unsigned)smax);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (s_cnt[0]) atomicAdd(&st->blk_count, (unsigned long long)s_cnt[0]);
+    if (s_cnt[1]) atomicMax(&stats->max_s, (int)s_cnt[1]);
   }
   // ---- the last CTA closes the block: budget, statistics, state of the next block's selection
   __threadfence();
@@ -1006,9 +1064,9 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     THANOS_CHECK_LAUNCH();
     tie_scan_kernel<<<1, 1024, 0, stream>>>(c, w.st, w.rowcnt, w.rowbase);
     THANOS_CHECK_LAUNCH();
-    int mg = (int)ceil_div(c, 8);
-    if (mg > NUM_SMS * 8) mg = NUM_SMS * 8;
-    mark_block_kernel<<<mg, 256, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
+    int mg = (int)ceil_div(c, MARK_WARPS);
+    if (mg > NUM_SMS * 2) mg = NUM_SMS * 2;
+    mark_block_kernel<<<mg, 32 * MARK_WARPS, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
                                               w.row_lists, w.list_counts, stats, r_ext);
     THANOS_CHECK_LAUNCH();
   } else {
