@@ -18,6 +18,7 @@ namespace thanos {
 namespace {
 
 constexpr int NB = 128;
+constexpr int PANEL_GROUP = 4;  // panels whose trailing updates go out as one product
 
 // ---- mean(diag H) -> lambda, xnorm ---------------------------------------------------------
 __global__ void __launch_bounds__(1024)
@@ -265,15 +266,19 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
     static std::atomic<unsigned long long> done{0};
     THANOS_CUDA(ensure_max_dyn_smem(diag_block_kernel, DIAG_SMEM, done));
   }
-  // ---- H_d = V V^T, panels from the last one backwards
-  for (int kb = nblk - 1; kb >= 0; --kb) {
-    const int k0 = kb * NB;
-    const int n = (b - k0 < NB) ? b - k0 : NB;
+  // ---- H_d = V V^T, panels from the last one backwards.  Full panels go in groups: a panel's
+  //      own 128 columns first receive, in one product, what the earlier panels of its group
+  //      owe them, and after the group's last panel a single product with K = 128 * (panels in
+  //      the group) updates everything to the left -- the trailing matrix is read and written
+  //      once per group instead of once per panel.
+  auto diag_block = [&](int k0, int n) -> thanos_status_t {
     diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(w.V, factor, w.Up, plane, b, k0, n,
-                                                       status_dev);
+                                                              status_dev);
     THANOS_CHECK_LAUNCH();
-    if (k0 == 0) break;
-    // V12 = A12 U22^T (rows above the block), written over A12 and as planes
+    return THANOS_OK;
+  };
+  // V12 = A12 U22^T for the rows above the block at k0, written over A12 and as planes
+  auto panel = [&](int k0, int n) -> thanos_status_t {
     THANOS_TRY(split3_planes(w.V + k0, b, k0, n, w.Vp + k0, b, plane, stream));
     TcGemmArgs g;
     g.D = w.V + k0;
@@ -292,26 +297,59 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
     g.N = n;
     g.K = n;
     g.status = w.tc_status;
-    THANOS_TRY(tc_gemm_split3(g, stream));
-    // A11 -= V12 V12^T on the tiles that touch the upper triangle
+    return tc_gemm_split3(g, stream);
+  };
+  // V[0:M, c0:c0+N] -= P P[c0:c0+N, :]^T with P = V12 panel columns [kc, kc + K): c0 = 0, N = M is
+  // the trailing update on the tiles that touch the upper triangle
+  auto downdate = [&](int M, int c0, int N, int kc, int K, int upper) -> thanos_status_t {
     TcGemmArgs y;
-    y.D = w.V;
+    y.D = w.V + c0;
     y.ldd = b;
-    y.A = w.Vp + k0;
+    y.A = w.Vp + kc;
     y.lda = b;
     y.a_plane = plane;
-    y.B = w.Vp + k0;
+    y.B = w.Vp + (int64_t)c0 * b + kc;
     y.ldb = b;
     y.b_plane = plane;
     y.b_kmajor = 1;
-    y.M = k0;
-    y.N = k0;
-    y.K = n;
+    y.M = M;
+    y.N = N;
+    y.K = K;
     y.alpha = -1.f;
     y.accumulate = 1;
-    y.upper_only = 1;
+    y.upper_only = upper;
     y.status = w.tc_status;
-    THANOS_TRY(tc_gemm_split3(y, stream));
+    return tc_gemm_split3(y, stream);
+  };
+  for (int kb = nblk - 1; kb >= 0;) {
+    const int k0 = kb * NB;
+    const int n = (b - k0 < NB) ? b - k0 : NB;
+    if (n < NB) {  // a ragged last panel goes alone
+      THANOS_TRY(diag_block(k0, n));
+      if (k0 == 0) break;
+      THANOS_TRY(panel(k0, n));
+      THANOS_TRY(downdate(k0, 0, k0, k0, n, 1));
+      kb -= 1;
+      continue;
+    }
+    int done = 0;
+    bool finished = false;  // the group reached the first panel
+    for (int j = 0; j < PANEL_GROUP; ++j) {
+      const int kj = k0 - j * NB;
+      // the panel's own columns first get what the group's earlier panels owe them
+      if (j > 0) THANOS_TRY(downdate(kj + NB, kj, NB, kj + NB, j * NB, 0));
+      THANOS_TRY(diag_block(kj, NB));
+      if (kj == 0) {
+        finished = true;
+        break;
+      }
+      THANOS_TRY(panel(kj, NB));
+      ++done;
+    }
+    if (finished) break;
+    const int kl = k0 - (done - 1) * NB;  // first column of the group
+    THANOS_TRY(downdate(kl, 0, kl, kl, done * NB, 1));
+    kb -= done;
   }
 
   // ---- U = inv(V) by halves: for the pair of diagonal blocks [r0, c0) and [c0, c0 + N),
