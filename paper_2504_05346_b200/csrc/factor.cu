@@ -41,18 +41,26 @@ diag_stats_kernel(const float* __restrict__ H, int b, float damp_rel, float* __r
   }
 }
 
-// V <- upper triangle of H (+ lambda on the diagonal); below the diagonal 0.
+// V <- upper triangle of H (+ lambda on the diagonal); below the diagonal 0.  Four columns per
+// thread (b is a multiple of 8, so every row starts on a 16-byte boundary).
 __global__ void copy_damped_upper_kernel(const float* __restrict__ H, float* __restrict__ V, int b,
                                          const float* __restrict__ lam) {
-  int j = blockIdx.x * blockDim.x + threadIdx.x;
-  int i = blockIdx.y;
+  const int j = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
+  const int i = blockIdx.y;
   if (j >= b) return;
-  float v = 0.f;
-  if (j >= i) {
-    v = H[(int64_t)i * b + j];
-    if (i == j) v += *lam;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (j + 3 >= i) {
+    v = *reinterpret_cast<const float4*>(H + (int64_t)i * b + j);
+    const float l = *lam;
+    if (j < i) v.x = 0.f;
+    if (j + 1 < i) v.y = 0.f;
+    if (j + 2 < i) v.z = 0.f;
+    if (j == i) v.x += l;
+    if (j + 1 == i) v.y += l;
+    if (j + 2 == i) v.z += l;
+    if (j + 3 == i) v.w += l;
   }
-  V[(int64_t)i * b + j] = v;
+  *reinterpret_cast<float4*>(V + (int64_t)i * b + j) = v;
 }
 
 // ---- diagonal block: A22 = V22 V22^T (V22 upper, i.e. Cholesky from the last row backwards) and
@@ -255,7 +263,7 @@ thanos_status_t prepare_inverse_impl(const float* H, int64_t b64, float damp_rel
 
   diag_stats_kernel<<<1, 1024, 0, stream>>>(H, b, damp_rel, xnorm, w.lam);
   THANOS_CHECK_LAUNCH();
-  dim3 cg((unsigned)ceil_div(b, 256), (unsigned)b);
+  dim3 cg((unsigned)ceil_div(b, 4 * 256), (unsigned)b);
   copy_damped_upper_kernel<<<cg, 256, 0, stream>>>(H, w.V, b, w.lam);
   THANOS_CHECK_LAUNCH();
   THANOS_CUDA(cudaMemsetAsync(factor, 0, (size_t)plane * sizeof(float), stream));
