@@ -364,21 +364,37 @@ __device__ __forceinline__ void select_pass_body(const float* __restrict__ Wc,
     const int wlog = st->wide ? WINDOW_LOG2_WIDE : WINDOW_LOG2;
     const unsigned WINDOW = 1u << wlog;
     const int WINDOW_SHIFT = wlog - WINDOW_BINS_LOG2;
-    for (int row = blockIdx.x; row < c; row += gridDim.x) {
-      const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-      // BR_UNROLL float4 loads in flight per thread: two when the working copy sits in L2, four
-      // when the residual streams from HBM
-      for (int q0 = threadIdx.x; q0 < w4; q0 += 256 * BR_UNROLL) {
-        float4 wv[BR_UNROLL], xv[BR_UNROLL];
+    // The residual is walked as one list of c * w4 16-byte items (row-major), 256 consecutive
+    // items per CTA and step, so that every thread has a load to issue whatever the width of the
+    // residual; a thread's (row, q) advances by the grid's stride without a division.
+    // BR_UNROLL loads in flight per thread: two when the working copy sits in L2, four when the
+    // residual streams from HBM.
+    const unsigned stride = gridDim.x * 256u;
+    const unsigned first = blockIdx.x * 256u + threadIdx.x;
+    const unsigned d_row = stride / (unsigned)w4, d_q = stride - d_row * (unsigned)w4;
+    unsigned row = first / (unsigned)w4, q = first - row * (unsigned)w4;
+    while (row < (unsigned)c) {
+      float4 wv[BR_UNROLL], xv[BR_UNROLL];
+      bool ok[BR_UNROLL];
 #pragma unroll
-        for (int u = 0; u < BR_UNROLL; ++u) {
-          const int q = q0 + 256 * u;
-          wv[u] = q < w4 ? wr[q] : make_float4(0.f, 0.f, 0.f, 0.f);
-          xv[u] = q < w4 ? __ldg(&xr[q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int u = 0; u < BR_UNROLL; ++u) {
+        ok[u] = row < (unsigned)c;
+        wv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        xv[u] = wv[u];
+        if (ok[u]) {
+          wv[u] = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1)[q];
+          xv[u] = __ldg(&xr[q]);
         }
+        row += d_row;
+        q += d_q;
+        if (q >= (unsigned)w4) {
+          q -= (unsigned)w4;
+          ++row;
+        }
+      }
 #pragma unroll
-        for (int u = 0; u < BR_UNROLL; ++u) {
-        if (q0 + 256 * u >= w4) break;
+      for (int u = 0; u < BR_UNROLL; ++u) {
+        if (!ok[u]) break;
         const float4 w = wv[u];
         const float4 x = xv[u];
         const unsigned k0 = metric_key(w.x, x.x), k1 = metric_key(w.y, x.y);
@@ -397,7 +413,6 @@ __device__ __forceinline__ void select_pass_body(const float* __restrict__ Wc,
               if (pos < (unsigned)CTA_CAND) s_cand[pos] = kk[e];
             }
           }
-        }
         }
       }
     }
