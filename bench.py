@@ -282,14 +282,14 @@ def roofline_by_kernel(trace_factor, trace_sweep, cfg, peaks, fp32_peak, masks, 
                 "bound": "hbm", "achieved": round(ach, 1), "peak": hbm, "unit": "GB/s",
                 "frac": round(ach / hbm, 4), "ms_per_step": round(ms, 3), "launches": n,
                 "work": "4 c (b - j1) bytes per block: one read of the residual"}
-    ms, n = t_of(trace_sweep, "tc_gemm_kernel")
+    ms, n = t_of(trace_sweep, "tc_gemm_")   # tc_gemm_kernel and tc_gemm_pair_kernel
     if ms:
         ach = 8.0 * upd_elems / (ms * 1e-3) / 1e9
         out["tc_gemm_kernel (sweep update)"] = {
             "bound": "hbm", "achieved": round(ach, 1), "peak": hbm, "unit": "GB/s",
             "frac": round(ach / hbm, 4), "ms_per_step": round(ms, 3), "launches": n,
             "work": "8 c (b - j2) bytes per block: the residual read and written once"}
-    ms, n = t_of(trace_factor, "tc_gemm_kernel")
+    ms, n = t_of(trace_factor, "tc_gemm_")
     if ms:
         flop = sum(k * (2.0 / 3.0) * float(b) ** 3 for b, k in n_inputs_by_b.items())
         ach = flop / (ms * 1e-3) / 1e12

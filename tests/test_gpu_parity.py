@@ -609,7 +609,10 @@ def test_host_buffer_entry_point_matches_device_path(T):
 # ------------------------------------------------------------------------------ dense product
 @pytest.mark.parametrize("M,N,K,bt", [
     (128, 128, 64, True), (128, 128, 64, False), (300, 520, 128, False), (300, 520, 128, True),
-    (64, 72, 8, False), (1000, 4096, 128, False), (257, 132, 200, True), (512, 384, 1024, True)])
+    (64, 72, 8, False), (1000, 4096, 128, False), (257, 132, 200, True), (512, 384, 1024, True),
+    # large enough for the CTA-pair kernel (256 x 256 tiles): ragged in M, N and K, the second
+    # CTA's half of the last tiles entirely outside the matrix; then a rank-128 update
+    (2688, 3712, 264, False), (2688, 3712, 264, True), (8192, 7168, 128, False)])
 def test_dense_product_matches_float64(T, M, N, K, bt):
     """The split-bf16 tensor-core product against a float64 product of the same fp32 inputs.
     Bound: a few units of 2^-24 of sum |a||b| per 16-term tensor-core accumulation step."""
