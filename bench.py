@@ -268,11 +268,21 @@ def roofline_by_kernel(trace_factor, trace_sweep, cfg, peaks, fp32_peak, masks, 
     B = cfg.B
     resid_elems = 0.0   # sum over layers and blocks of c (b - j1): one look at the residual per block
     upd_elems = 0.0     # sum over layers and blocks of c (b - j2): what a block's update changes
+    grouped_layers = 0
     for L in cfg.layers:
+        # n:m sweeps of wide layers update in groups of 512 columns: a block's update reaches the
+        # rest of its group at once, the columns to the right of the group once per group
+        group = 1
+        if not unstructured and L.b >= 2048 and B < 512:
+            group = max(1, min(8, 512 // B))
+            grouped_layers += 1
         for j1 in range(0, L.b, B):
             j2 = min(L.b, j1 + B)
             resid_elems += float(L.c) * (L.b - j1)
-            upd_elems += float(L.c) * (L.b - j2)
+            ge = min(L.b, (j1 // (group * B) + 1) * group * B)   # end of the block's group
+            upd_elems += float(L.c) * (ge - j2)
+            if j2 == ge:
+                upd_elems += float(L.c) * (L.b - ge)
     hbm = peaks["hbm_gbs"]
     if unstructured:
         ms, n = t_of(trace_sweep, "::select_")   # select_pass_kernel and select_rest_kernel
@@ -288,7 +298,19 @@ def roofline_by_kernel(trace_factor, trace_sweep, cfg, peaks, fp32_peak, masks, 
         out["tc_gemm_kernel (sweep update)"] = {
             "bound": "hbm", "achieved": round(ach, 1), "peak": hbm, "unit": "GB/s",
             "frac": round(ach / hbm, 4), "ms_per_step": round(ms, 3), "launches": n,
-            "work": "8 c (b - j2) bytes per block: the residual read and written once"}
+            "work": "8 bytes per weight an update changes: c (b - j2) per block; in n:m sweeps of "
+                    "wide layers c (group end - j2) per block and c (b - group end) per group "
+                    "of 512 columns"}
+        if grouped_layers:
+            # with K = 512 per group the update is a tensor-bound product: also against that bound
+            flop = sum(float(L.c) * float(L.b) * float(L.b) for L in cfg.layers)   # 2 c B (b - j2) / block
+            tf = flop / (ms * 1e-3) / 1e12
+            pk = peaks["bf16_tflops_sustained"]
+            out["tc_gemm_kernel (sweep update)"].update({
+                "tensor_useful_tflops": round(tf, 1), "tensor_frac_useful": round(tf / pk, 4),
+                "tensor_frac_executed": round(6.0 * tf / pk, 4),
+                "tensor_note": "c b^2 useful FLOP per layer; the kernel executes six bf16-plane "
+                               "products per fp32 product"})
     ms, n = t_of(trace_factor, "tc_gemm_")
     if ms:
         flop = sum(k * (2.0 / 3.0) * float(b) ** 3 for b, k in n_inputs_by_b.items())

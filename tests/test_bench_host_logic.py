@@ -56,3 +56,26 @@ def test_mode_selection_of_a_configuration():
     alt = bench.select_mode(cfg, 1)
     assert alt.mode == "unstructured" and abs(alt.p - 0.6) < 1e-12 and alt.layers == cfg.layers
     assert bench.short_kernel_name("void thanos::(anonymous namespace)::foo_kernel<2>(int)") == "foo_kernel<2>"
+
+
+def test_update_bytes_of_a_grouped_nm_sweep():
+    """n:m sweeps of layers at least 2048 wide update in groups of 512 columns: the bytes an update
+    changes are counted per group to the right of it, and the product is also rated as tensor work."""
+    cfg = WL.CONFIGS["llama2_70b"]   # 2:4, B = 128: groups of four blocks
+    assert cfg.mode == "nm" and cfg.B == 128
+    peaks = {"hbm_gbs": 1000.0, "bf16_tflops": 100.0, "bf16_tflops_sustained": 80.0}
+    tr_s = {"thanos::(anonymous namespace)::tc_gemm_pair_kernel(...)": [5, 1.0],
+            "thanos::(anonymous namespace)::tc_gemm_kernel(...)": [5, 1.0]}
+    out = bench.roofline_by_kernel({}, tr_s, cfg, peaks, 50.0, [], {})
+    want = 0.0
+    for L in cfg.layers:
+        for j1 in range(0, L.b, 128):
+            j2 = min(L.b, j1 + 128)
+            ge = min(L.b, (j1 // 512 + 1) * 512)
+            want += L.c * (ge - j2) + (L.c * (L.b - ge) if j2 == ge else 0)
+    e = out["tc_gemm_kernel (sweep update)"]
+    assert e["launches"] == 10 and abs(e["ms_per_step"] - 2.0) < 1e-9   # both kernels counted
+    assert abs(e["achieved"] - 8.0 * want / 2e-3 / 1e9) / e["achieved"] < 1e-3
+    flop = sum(float(L.c) * L.b * L.b for L in cfg.layers)
+    assert abs(e["tensor_useful_tflops"] - flop / 2e-3 / 1e12) / e["tensor_useful_tflops"] < 1e-3
+    assert abs(e["tensor_frac_executed"] - 6.0 * e["tensor_frac_useful"]) < 1e-3
