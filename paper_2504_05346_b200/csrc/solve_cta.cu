@@ -6,12 +6,14 @@
 // B = 256 (128 unknowns).  The gathered
 // matrix lives in shared memory as the lower triangle of 16 x 16 tiles (1 KB each, 16-byte chunks
 // swizzled by the row so that the accesses below are free of bank conflicts); the right-hand
-// side is appended as row n, so that the factorisation L L^T also yields y = L^{-1} rhs.
+// side is a vector of its own (as a row of the matrix it would cost a whole extra tile row
+// whenever the system size is a multiple of 16, which it always is for n:m masks).
 // Right-looking tile Cholesky by the CTA's warps (16, or 4 for the smaller systems; with 16 warps
 // the trailing update runs on the tensor cores from bf16 planes of the panel, see below): panel solve (one thread per row), trailing update
 // (one warp per target tile, handed out by a shared counter); warp 0 updates and factors the
 // next diagonal tile first, which takes the only serial step off the critical path.  Blocked
-// back substitution L^T x = y, then the change of the block's weights as in the small kernel.
+// substitutions L y = rhs and L^T x = y, then the change of the block's weights as in the small
+// kernel.
 #include "common.cuh"
 #include "tile_ops.cuh"
 
@@ -24,7 +26,7 @@ using tile::elem_off;
 using tile::tile_update;
 
 constexpr unsigned FULL = 0xffffffffu;
-constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 - 1 = 319 unknowns
+constexpr int MAX_TILES = 20;  // tile rows: systems of up to 16 * 20 = 320 unknowns (319 are handed out)
 
 // tile (I, J), J <= I, of the lower triangle; 256 floats each
 __device__ __forceinline__ int tile_base(int I, int J) { return (((I * (I + 1)) >> 1) + J) << 8; }
@@ -195,6 +197,29 @@ __device__ __forceinline__ void macro_update_mma(float* __restrict__ A, int K, i
     }
 }
 
+// The same 2 x 2 group without stored planes: the fp32 panel tiles are split into bf16 planes in
+// registers (tile_ops.cuh), so a group costs four fragment loads, 48 tensor-core instructions and
+// the read-modify-write of its targets.  For the four-warp CTAs, whose shared memory has no room
+// for the planes of a panel.
+__device__ __forceinline__ void macro_update_frag(float* __restrict__ A, int K, int I0, int J0, int T,
+                                                  unsigned vmask, const tile::FragOff& fo) {
+  const int I1 = I0 + 1 < T ? I0 + 1 : T - 1, J1 = J0 + 1 < T ? J0 + 1 : T - 1;
+  tile::PanelFrag fa[2], fb[2];
+  tile::load_panel_frag(A + tile_base(I0, K), fo, fa[0]);
+  tile::load_panel_frag(A + tile_base(I1, K), fo, fa[1]);
+  tile::load_panel_frag(A + tile_base(J0, K), fo, fb[0]);
+  tile::load_panel_frag(A + tile_base(J1, K), fo, fb[1]);
+#pragma unroll
+  for (int di = 0; di < 2; ++di)
+#pragma unroll
+    for (int dj = 0; dj < 2; ++dj) {
+      if (!(vmask & (1u << (2 * di + dj)))) continue;  // warp-uniform
+      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      tile::frag_product(acc, fa[di], fb[dj]);
+      tile::tile_subtract(A + tile_base(I0 + di, J0 + dj), acc, fo);
+    }
+}
+
 // exclusive prefix sum of one value per thread over the CTA
 template <int CTA_WARPS>
 __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* warp_sums,
@@ -228,7 +253,7 @@ __device__ __forceinline__ unsigned cta_exclusive_scan(unsigned x, unsigned* war
 // four rows in flight with four warps each beat both one row with sixteen warps and the
 // warp-per-row kernel (whose 41 KB per warp leave room for five rows per SM).
 template <int CTA_THREADS>
-__global__ void __launch_bounds__(CTA_THREADS, 512 / CTA_THREADS)
+__global__ void __launch_bounds__(CTA_THREADS, CTA_THREADS == 128 ? 5 : 512 / CTA_THREADS)
 solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
                       const float* __restrict__ Gm, const float* __restrict__ Sm, int ld_mat,
                       __nv_bfloat16* __restrict__ D, int64_t dplane, int c, int b, int j1, int Bw,
@@ -255,6 +280,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
   __nv_bfloat16* Pp = reinterpret_cast<__nv_bfloat16*>(
       dyn + ((reinterpret_cast<unsigned char*>(scratch + 48) - dyn + 15) & ~(size_t)15));
   const int plane_stride = 16 * (tiles - 1) * PLANE_LD;
+  const tile::FragOff frag_off = tile::make_frag_off(lane >> 2, lane & 3);
 
   int cnt0, cnt1;
   if (row_lists) {
@@ -303,8 +329,8 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       sel[n + tid] = 0;
       oth[no + tid] = 0;
     }
-    const int T = (n + 16) >> 4;   // tile rows of the system plus the right-hand-side row
-    const int Tf = (n + 15) >> 4;  // tile columns that are factored
+    const int T = (n + 15) >> 4;   // tile rows (= tile columns) of the system
+    const int Tf = T;
     if ((s > t) != kpath || T > tiles) {
       // cannot happen for lists and launch sizes made by this library
       if (tid == 0) report_error(&stats->status, THANOS_ERR_SHAPE, row);
@@ -336,7 +362,7 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       rhsv[e] = g;
     }
     __syncthreads();
-    // ---- gather the lower triangle of M[sel, sel], the right-hand-side row n, identity padding
+    // ---- gather the lower triangle of M[sel, sel], identity padding
     {
       // A tile has 256 entries: with 512 threads two tiles are filled at a time, with 128 threads
       // a thread fills two entries of each tile; eight tiles' loads are in flight per thread.
@@ -364,8 +390,6 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
               x = 0.f;
             else if (i < n)
               x = j < n ? __ldg(M + (int)sel[i] * ld_mat + (int)sel[j]) : 0.f;
-            else if (i == n)
-              x = j < n ? rhsv[j] : (j == n ? 1.f : 0.f);
             else
               x = i == j ? 1.f : 0.f;
             v[u][h] = x;
@@ -387,12 +411,31 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
     }
     __syncthreads();
     bool bad = false;
-    if (warp == 0) bad = tile::factor_diag_tile<false>(A + tile_base(0, 0), invd, 0, n, lane) >= 0;
+    if (warp == 0 && T > 0) bad = tile::factor_diag_tile<false>(A + tile_base(0, 0), invd, 0, n, lane) >= 0;
+    for (int i = tid; i < 16 * T + 4; i += CTA_THREADS) xs[i] = i < n ? rhsv[i] : 0.f;
     __syncthreads();
-    // ---- right-looking tile Cholesky
+    // ---- right-looking tile Cholesky; the forward substitution L y = rhs rides along: tile
+    //      column K of y is solved by the last warp at the start of step K (L_KK is factored and
+    //      xs[16 K ..] has received every earlier column by then), and the entries below it are
+    //      updated with the solved panel at the start of the trailing phase
     for (int K = 0; K < Tf; ++K) {
       const int m = T - K - 1;  // tile rows below the diagonal tile
       if (tid == 0) *s_counter = 0;
+      if (warp == CTA_THREADS / 32 - 1) {
+        const float* Lk = A + tile_base(K, K);
+        const int me = 16 * K + (lane & 15);
+        float res = me < n ? xs[me] : 0.f;
+#pragma unroll
+        for (int w = 0; w < 16; ++w) {
+          const int idx = 16 * K + w;
+          float yi = __shfl_sync(FULL, res, w);
+          yi = idx < n ? yi * invd[idx] : 0.f;
+          const float lkw = Lk[elem_off(lane & 15, w)];
+          if ((lane & 15) > w) res = fmaf(-lkw, yi, res);
+          if ((lane & 15) == w) res = yi;
+        }
+        if (lane < 16 && me < n) xs[me] = res;
+      }
       // panel: X L_KK^T = A_IK for the rows below, one thread per row
       {
         const float* Lk = A + tile_base(K, K);
@@ -403,6 +446,15 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
         }
       }
       __syncthreads();
+      // right-hand side below tile row K: xs[k] -= L[k, 16 K ..] y_K
+      for (int k = 16 * (K + 1) + tid; k < 16 * T; k += CTA_THREADS) {
+        const float* Lt = A + tile_base(k >> 4, K);
+        const int kk = k & 15;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < 16; ++w) acc = fmaf(Lt[elem_off(kk, w)], xs[16 * K + w], acc);
+        xs[k] -= acc;
+      }
       // trailing update; warp 0 first brings the next diagonal tile up to date and factors it
       if (warp == 0 && K + 1 < Tf) {
         float* Ct = A + tile_base(K + 1, K + 1);
@@ -438,6 +490,8 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
           if (vmask) {
             if (use_planes)
               macro_update_mma(A, K, I0, J0, T, vmask, Pp, plane_stride, lane);
+            else if (CTA_THREADS == 128)
+              macro_update_frag(A, K, I0, J0, T, vmask, frag_off);
             else
               macro_update(A, K, I0, J0, T, vmask, lane);
           }
@@ -446,18 +500,13 @@ solve_rows_cta_kernel(float* __restrict__ Wc, const uint8_t* __restrict__ mask,
       __syncthreads();
     }
     if (warp == 0 && bad && lane == 0) *s_bad = 1;
-    // ---- y = row n of L; blocked back substitution L^T x = y from the bottom
-    {
-      const int In = n >> 4, rn = n & 15;
-      for (int i = tid; i < 16 * T + 4; i += CTA_THREADS)
-        xs[i] = i < n ? A[tile_base(In, i >> 4) + elem_off(rn, i & 15)] : 0.f;
-    }
     __syncthreads();
     if (*s_bad) {
       if (tid == 0) report_error(&stats->status, THANOS_ERR_NOT_SPD, row);
       for (int jj = tid; jj < Bw; jj += CTA_THREADS) store_split3(D + (int64_t)row * ldd + jj, dplane, 0.f);
       continue;
     }
+    // ---- blocked back substitution L^T x = y from the bottom
     for (int Kb = Tf - 1; Kb >= 0; --Kb) {
       if (warp == 0) {
         const float* Lk = A + tile_base(Kb, Kb);
@@ -532,7 +581,14 @@ thanos_status_t launch_cta_solve_t(float* Wc, const uint8_t* mask, const float* 
     static std::atomic<unsigned long long> done{0};
     THANOS_CUDA(ensure_max_dyn_smem(solve_rows_cta_kernel<CTA_THREADS>, 227 * 1024, done));
   }
-  const int ctas = NUM_SMS * (512 / CTA_THREADS);
+  // CTAs per SM: what the shared memory of a CTA (plus the 1 KB the system keeps per CTA) allows,
+  // up to five of the four-warp CTAs
+  int per_sm = 512 / CTA_THREADS;
+  if (CTA_THREADS == 128) {
+    per_sm = (int)((228 * 1024) / (smem + 1024));
+    per_sm = per_sm < 1 ? 1 : (per_sm > 5 ? 5 : per_sm);
+  }
+  const int ctas = NUM_SMS * per_sm;
   const int grid = c < ctas ? c : ctas;
   solve_rows_cta_kernel<CTA_THREADS><<<(unsigned)grid, CTA_THREADS, smem, stream>>>(
       Wc, mask, G, S, ld_mat, D, dplane, c, b, j1, Bw, ldd, tiles, row_lists, list_counts,
@@ -546,7 +602,7 @@ thanos_status_t launch_cta_solve(float* Wc, const uint8_t* mask, const float* G,
                                  int Bw, int ldd, int n_max, const int* row_lists,
                                  const unsigned* list_counts, int fixed_kind, int report_max_s,
                                  thanos_stats_t* stats, cudaStream_t stream) {
-  const int tiles = (n_max + 16) / 16;
+  const int tiles = (n_max + 15) / 16 > 0 ? (n_max + 15) / 16 : 1;
   if (tiles > MAX_TILES || Bw > 1024) return THANOS_ERR_SHAPE;
   const size_t smem = cta_smem_bytes(tiles, Bw);
   if (smem > 227 * 1024) return THANOS_ERR_SHAPE;

@@ -127,5 +127,95 @@ __device__ __forceinline__ void panel_row_solve(float* arow_tile, int r, const f
         make_float4(x[4 * cc], x[4 * cc + 1], x[4 * cc + 2], x[4 * cc + 3]);
 }
 
+// ---- tile products on the tensor cores (mma.sync m16n8k16): fp32 tiles are split into three
+// bf16 planes in registers (24 significant bits) and six plane products are accumulated in fp32.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+  // no side effects beyond its outputs: not volatile, so that independent chains interleave
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// (x0, x1) -> three words of two bf16 each (x0 in the low half): x = p0 + p1 + p2 to 24 bits
+__device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& p0, uint32_t& p1,
+                                           uint32_t& p2) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  p0 = *reinterpret_cast<const uint32_t*>(&h);
+  x0 -= __uint_as_float(p0 << 16);
+  x1 -= __uint_as_float(p0 & 0xffff0000u);
+  h = __floats2bfloat162_rn(x0, x1);
+  p1 = *reinterpret_cast<const uint32_t*>(&h);
+  x0 -= __uint_as_float(p1 << 16);
+  x1 -= __uint_as_float(p1 & 0xffff0000u);
+  h = __floats2bfloat162_rn(x0, x1);
+  p2 = *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Fragment of a 16 x 16 panel tile P for mma.m16n8k16 (g = lane / 4, t = lane % 4): word 0 rows g,
+// columns 2t, 2t + 1; word 1 row g + 8; words 2, 3 the same rows, columns 2t + 8, 2t + 9.  As the A
+// operand (P itself) all four words are used; as the B operand (P^T) half h of the 8-wide column
+// blocks takes words h and h + 2.
+struct PanelFrag {
+  uint32_t w[3][4];
+};
+// Offsets of a lane's four fragment words inside any tile (they depend on the lane only): word
+// 2 h' + h'' is row g + 8 h'', columns 2t + 8 h' -- also the lane's accumulator entries of column
+// half h'.
+struct FragOff {
+  int o[4];
+};
+__device__ __forceinline__ FragOff make_frag_off(int g, int t) {
+  FragOff f;
+  f.o[0] = elem_off(g, 2 * t);
+  f.o[1] = elem_off(g + 8, 2 * t);
+  f.o[2] = elem_off(g, 2 * t + 8);
+  f.o[3] = elem_off(g + 8, 2 * t + 8);
+  return f;
+}
+__device__ __forceinline__ void load_panel_frag(const float* __restrict__ Tt, const FragOff& fo,
+                                                PanelFrag& f) {
+  const float2 v0 = *reinterpret_cast<const float2*>(Tt + fo.o[0]);
+  const float2 v1 = *reinterpret_cast<const float2*>(Tt + fo.o[1]);
+  const float2 v2 = *reinterpret_cast<const float2*>(Tt + fo.o[2]);
+  const float2 v3 = *reinterpret_cast<const float2*>(Tt + fo.o[3]);
+  split_pair(v0.x, v0.y, f.w[0][0], f.w[1][0], f.w[2][0]);
+  split_pair(v1.x, v1.y, f.w[0][1], f.w[1][1], f.w[2][1]);
+  split_pair(v2.x, v2.y, f.w[0][2], f.w[1][2], f.w[2][2]);
+  split_pair(v3.x, v3.y, f.w[0][3], f.w[1][3], f.w[2][3]);
+}
+
+// acc[h] += P_a P_b^T (the two 8-column halves h) from the six plane products, smallest first
+__device__ __forceinline__ void frag_product(float (&acc)[2][4], const PanelFrag& fa,
+                                             const PanelFrag& fb) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    mma_bf16_16816(acc[h], fa.w[1], fb.w[1][h], fb.w[1][h + 2]);  // m m
+    mma_bf16_16816(acc[h], fa.w[2], fb.w[0][h], fb.w[0][h + 2]);  // l h
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[2][h], fb.w[2][h + 2]);  // h l
+    mma_bf16_16816(acc[h], fa.w[1], fb.w[0][h], fb.w[0][h + 2]);  // m h
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[1][h], fb.w[1][h + 2]);  // h m
+    mma_bf16_16816(acc[h], fa.w[0], fb.w[0][h], fb.w[0][h + 2]);  // h h
+  }
+}
+
+// C -= acc for one target tile (accumulator layout: rows g, g + 8, columns 8 h + 2 t, + 1)
+__device__ __forceinline__ void tile_subtract(float* __restrict__ Ct, const float (&acc)[2][4],
+                                              const FragOff& fo) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float2* c0 = reinterpret_cast<float2*>(Ct + fo.o[2 * h]);
+    float2* c1 = reinterpret_cast<float2*>(Ct + fo.o[2 * h + 1]);
+    float2 u0 = *c0, u1 = *c1;
+    u0.x -= acc[h][0];
+    u0.y -= acc[h][1];
+    u1.x -= acc[h][2];
+    u1.y -= acc[h][3];
+    *c0 = u0;
+    *c1 = u1;
+  }
+}
+
 }  // namespace tile
 }  // namespace thanos
