@@ -735,7 +735,7 @@ def run_single_layer(args):
     B_.build()
     T.load_library()
     c, b, a = [int(v) for v in args.single_layer.split(",")]
-    cfg = WL.CONFIGS[args.workload]
+    cfg = select_mode(WL.CONFIGS[args.workload], args.mode_index)
     if args.block > 0:
         cfg = dataclasses.replace(cfg, B=args.block)
     dev = torch.device("cuda", 0)

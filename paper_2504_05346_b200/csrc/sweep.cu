@@ -72,6 +72,7 @@ struct SweepState {
   unsigned int cand_total;       // keys the bracket pass copied out of its window
   int cand_overflow;             // the copy did not fit: the refine pass rescans the residual
   int wide;                      // a bracket missed in this sweep: use the wide window
+  int tie_in_block;              // an entry equal to the threshold lies in the current block's columns
 };
 
 __device__ __forceinline__ unsigned metric_key(float w, float xn) {
@@ -308,6 +309,7 @@ __device__ __forceinline__ void select_pass_body(const float* __restrict__ Wc,
   if (phase == PH_DONE && !first_launch) return;
   if (first_launch && blockIdx.x == 0 && threadIdx.x == 0) {
     list_counts[0] = list_counts[1] = 0;
+    st->tie_in_block = 0;
     if (r_ext) st->r = *r_ext;
   }
   const int lane = threadIdx.x & 31;
@@ -565,22 +567,42 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
 
 // The passes a block may still need after its first two launches (bracket + refine, or the first
 // two radix passes): up to three more radix passes, in ONE cooperative launch with a grid barrier
-// between them.  It returns at once when the threshold is known, which is the usual case, so a
-// block step carries one launch that does nothing instead of three.
+// between them.  With the threshold known on entry, which is the usual case, it runs none of
+// them, so a block step carries one nearly idle launch instead of three.  Last it finds out
+// whether the order of tied entries can matter to this block's mask at all.
 template <int BR_UNROLL>
 __global__ void __launch_bounds__(256)
 select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
-                   int j1, SweepState* st, unsigned* __restrict__ hist,
+                   int j1, int Bw, SweepState* st, unsigned* __restrict__ hist,
                    unsigned* __restrict__ list_counts, thanos_stats_t* stats,
                    unsigned* __restrict__ cand, unsigned cand_cap) {
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
   for (int it = 0; it < 3; ++it) {
     // the phase only changes between two grid barriers, so every CTA reads the same value
-    if (*reinterpret_cast<volatile int*>(&st->phase) == PH_DONE) return;
+    if (*reinterpret_cast<volatile int*>(&st->phase) == PH_DONE) break;
     select_pass_body<BR_UNROLL>(Wc, xnorm, c, b, j1, st, hist, nullptr, list_counts, 0, stats, cand,
                                 cand_cap);
     grid.sync();
   }
+  // The threshold is final.  When only some of the entries equal to it are removed, their order
+  // over the whole residual decides which -- but that only matters to this block's mask if one
+  // of them lies in the block's own columns.  Look there (c * Bw entries) before anyone counts
+  // ties over the whole residual.
+  volatile SweepState* vs = st;
+  if (vs->none || vs->need_eq == vs->count_eq) return;
+  const unsigned tau = vs->tau;
+  const int w4 = Bw >> 2;
+  const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
+  int found = 0;
+  const unsigned total = (unsigned)c * (unsigned)w4;
+  for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total; i += gridDim.x * 256u) {
+    const unsigned row = i / (unsigned)w4, q = i - row * (unsigned)w4;
+    const float4 w = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1)[q];
+    const float4 x = __ldg(&xr[q]);
+    found |= (metric_key(w.x, x.x) == tau) | (metric_key(w.y, x.y) == tau) |
+             (metric_key(w.z, x.z) == tau) | (metric_key(w.w, x.w) == tau);
+  }
+  if (__syncthreads_or(found) && threadIdx.x == 0) st->tie_in_block = 1;
 }
 
 // Rows' counts of entries equal to the threshold over the residual (only needed when the
@@ -588,7 +610,7 @@ select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
 __global__ void __launch_bounds__(256)
 tie_count_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                  int j1, const SweepState* __restrict__ st, unsigned* __restrict__ rowcnt) {
-  if (st->none || st->need_eq == st->count_eq) return;
+  if (st->none || st->need_eq == st->count_eq || !st->tie_in_block) return;
   __shared__ unsigned red[8];
   const unsigned tau = st->tau;
   const int w4 = (b - j1) >> 2;
@@ -618,7 +640,7 @@ tie_count_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, 
 __global__ void __launch_bounds__(1024)
 tie_scan_kernel(int c, const SweepState* __restrict__ st, const unsigned* __restrict__ rowcnt,
                 unsigned long long* __restrict__ rowbase) {
-  if (st->none || st->need_eq == st->count_eq) return;
+  if (st->none || st->need_eq == st->count_eq || !st->tie_in_block) return;
   __shared__ unsigned long long wsum[32];
   __shared__ unsigned long long carry;
   if (threadIdx.x == 0) carry = 0;
@@ -668,6 +690,7 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
   const bool none = st->none != 0;
   const unsigned tau = st->tau;
   const bool all_ties = st->need_eq == st->count_eq;
+  const bool tie_in_block = st->tie_in_block != 0;  // else no entry of the block equals the threshold
   const unsigned long long need = st->need_eq;
   unsigned long long total = 0;
   int smax = 0;
@@ -676,7 +699,7 @@ mark_block_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm,
     if (threadIdx.x < 2) s_cnt[threadIdx.x] = 0;
     __syncthreads();
     if (row < c) {
-    unsigned long long rank = (none || all_ties) ? 0ull : rowbase[row];
+    unsigned long long rank = (none || all_ties || !tie_in_block) ? 0ull : rowbase[row];
     int s = 0;
     // a lane takes four consecutive columns (Bw % 8 == 0): one 16-byte load of the weights, one of
     // the norms and one 4-byte store of mask bytes per 128 columns
@@ -1060,14 +1083,15 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
       // whatever is left of a radix route, behind grid barriers (sg2 <= 2 CTAs per SM: co-resident)
       const float* a_Wc = Wc;
       const float* a_xn = xnorm;
-      int a_c = c, a_b = b, a_j1 = j1;
+      int a_c = c, a_b = b, a_j1 = j1, a_bw = Bw;
       SweepState* a_st = w.st;
       unsigned* a_hist = w.hist;
       unsigned* a_lc = w.list_counts;
       thanos_stats_t* a_stats = stats;
       unsigned* a_cand = w.cand;
       unsigned a_cap = (unsigned)w.cand_cap;
-      void* args[] = {&a_Wc, &a_xn, &a_c, &a_b, &a_j1, &a_st, &a_hist, &a_lc, &a_stats, &a_cand, &a_cap};
+      void* args[] = {&a_Wc, &a_xn, &a_c, &a_b, &a_j1, &a_bw, &a_st, &a_hist, &a_lc, &a_stats, &a_cand,
+                      &a_cap};
       const void* fn = big ? reinterpret_cast<const void*>(&select_rest_kernel<4>)
                            : reinterpret_cast<const void*>(&select_rest_kernel<2>);
       if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)sg2), dim3(256), args, 0, stream) !=
