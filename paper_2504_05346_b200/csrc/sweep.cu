@@ -565,17 +565,76 @@ select_pass_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
                               cand, cand_cap);
 }
 
+// Rows' counts of entries equal to the threshold over the residual (only needed when the
+// tie-break has to leave some of them unpruned and one of them lies in the block): a CTA takes
+// rows blockIdx.x, blockIdx.x + gridDim.x, ...  256 threads per CTA.
+__device__ __forceinline__ void tie_count_rows(const float* __restrict__ Wc,
+                                               const float* __restrict__ xnorm, int c, int b, int j1,
+                                               unsigned tau, unsigned* __restrict__ rowcnt) {
+  __shared__ unsigned red[8];
+  const int w4 = (b - j1) >> 2;
+  for (int row = blockIdx.x; row < c; row += gridDim.x) {
+    const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
+    const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
+    unsigned cnt = 0;
+#pragma unroll 4
+    for (int q = threadIdx.x; q < w4; q += 256) {
+      float4 w = wr[q];
+      float4 x = __ldg(&xr[q]);
+      cnt += (metric_key(w.x, x.x) == tau) + (metric_key(w.y, x.y) == tau) +
+             (metric_key(w.z, x.z) == tau) + (metric_key(w.w, x.w) == tau);
+    }
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned t = 0;
+      for (int i = 0; i < 8; ++i) t += red[i];
+      rowcnt[row] = t;
+    }
+    __syncthreads();
+  }
+}
+
+// rowbase[row] = number of tied entries in the rows before it (exclusive scan by one CTA of 256).
+__device__ __forceinline__ void tie_scan_rows(int c, const unsigned* __restrict__ rowcnt,
+                                              unsigned long long* __restrict__ rowbase) {
+  __shared__ unsigned long long wsum[8];
+  __shared__ unsigned long long carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < c; base += 256) {
+    const int row = base + threadIdx.x;
+    const unsigned long long v = row < c ? __ldcg(&rowcnt[row]) : 0;
+    unsigned long long inc = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long u = __shfl_up_sync(0xffffffffu, inc, o);
+      if ((threadIdx.x & 31) >= o) inc += u;
+    }
+    if ((threadIdx.x & 31) == 31) wsum[threadIdx.x >> 5] = inc;
+    __syncthreads();
+    unsigned long long before = carry;
+    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before += wsum[w];
+    const unsigned long long excl = before + inc - v;
+    if (row < c) rowbase[row] = excl;
+    __syncthreads();
+    if (threadIdx.x == 255) carry = excl + v;
+    __syncthreads();
+  }
+}
+
 // The passes a block may still need after its first two launches (bracket + refine, or the first
 // two radix passes): up to three more radix passes, in ONE cooperative launch with a grid barrier
 // between them.  With the threshold known on entry, which is the usual case, it runs none of
 // them, so a block step carries one nearly idle launch instead of three.  Last it finds out
-// whether the order of tied entries can matter to this block's mask at all.
+// whether the order of tied entries can matter to this block's mask at all, and ranks them if so.
 template <int BR_UNROLL>
 __global__ void __launch_bounds__(256)
 select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
                    int j1, int Bw, SweepState* st, unsigned* __restrict__ hist,
                    unsigned* __restrict__ list_counts, thanos_stats_t* stats,
-                   unsigned* __restrict__ cand, unsigned cand_cap) {
+                   unsigned* __restrict__ cand, unsigned cand_cap,
+                   unsigned* __restrict__ rowcnt, unsigned long long* __restrict__ rowbase) {
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
   for (int it = 0; it < 3; ++it) {
     // the phase only changes between two grid barriers, so every CTA reads the same value
@@ -603,73 +662,13 @@ select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
              (metric_key(w.z, x.z) == tau) | (metric_key(w.w, x.w) == tau);
   }
   if (__syncthreads_or(found) && threadIdx.x == 0) st->tie_in_block = 1;
-}
-
-// Rows' counts of entries equal to the threshold over the residual (only needed when the
-// tie-break has to leave some of them unpruned).
-__global__ void __launch_bounds__(256)
-tie_count_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
-                 int j1, const SweepState* __restrict__ st, unsigned* __restrict__ rowcnt) {
-  if (st->none || st->need_eq == st->count_eq || !st->tie_in_block) return;
-  __shared__ unsigned red[8];
-  const unsigned tau = st->tau;
-  const int w4 = (b - j1) >> 2;
-  for (int row = blockIdx.x; row < c; row += gridDim.x) {
-    const float4* wr = reinterpret_cast<const float4*>(Wc + (int64_t)row * b + j1);
-    const float4* xr = reinterpret_cast<const float4*>(xnorm + j1);
-    unsigned cnt = 0;
-#pragma unroll 4
-    for (int q = threadIdx.x; q < w4; q += 256) {
-      float4 w = wr[q];
-      float4 x = __ldg(&xr[q]);
-      cnt += (metric_key(w.x, x.x) == tau) + (metric_key(w.y, x.y) == tau) +
-             (metric_key(w.z, x.z) == tau) + (metric_key(w.w, x.w) == tau);
-    }
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = cnt;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      unsigned t = 0;
-      for (int i = 0; i < 8; ++i) t += red[i];
-      rowcnt[row] = t;
-    }
-    __syncthreads();
-  }
-}
-
-__global__ void __launch_bounds__(1024)
-tie_scan_kernel(int c, const SweepState* __restrict__ st, const unsigned* __restrict__ rowcnt,
-                unsigned long long* __restrict__ rowbase) {
-  if (st->none || st->need_eq == st->count_eq || !st->tie_in_block) return;
-  __shared__ unsigned long long wsum[32];
-  __shared__ unsigned long long carry;
-  if (threadIdx.x == 0) carry = 0;
-  __syncthreads();
-  for (int base = 0; base < c; base += 1024) {
-    int row = base + threadIdx.x;
-    unsigned long long v = row < c ? rowcnt[row] : 0;
-    unsigned long long inc = v;
-    for (int o = 1; o < 32; o <<= 1) {
-      unsigned long long u = __shfl_up_sync(0xffffffffu, inc, o);
-      if ((threadIdx.x & 31) >= o) inc += u;
-    }
-    if ((threadIdx.x & 31) == 31) wsum[threadIdx.x >> 5] = inc;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      unsigned long long t = wsum[threadIdx.x], s = t;
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned long long u = __shfl_up_sync(0xffffffffu, s, o);
-        if (threadIdx.x >= o) s += u;
-      }
-      wsum[threadIdx.x] = s - t;
-    }
-    __syncthreads();
-    unsigned long long excl = carry + wsum[threadIdx.x >> 5] + inc - v;
-    if (row < c) rowbase[row] = excl;
-    __syncthreads();
-    if (threadIdx.x == 1023) carry = excl + v;
-    __syncthreads();
-  }
+  grid.sync();
+  if (!vs->tie_in_block) return;
+  // It does: rank the tied entries in (row, column) order -- their count per row over the whole
+  // residual, then the exclusive scan over the rows that the mask kernel reads.
+  tie_count_rows(Wc, xnorm, c, b, j1, tau, rowcnt);
+  grid.sync();
+  if (blockIdx.x == 0) tie_scan_rows(c, rowcnt, rowbase);
 }
 
 // One warp per row: set the block's mask bytes.  key < tau -> removed; key == tau -> removed
@@ -1057,10 +1056,6 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
   if (upd_end < 0) upd_end = b;
   int s_fixed = -1;
   if (mode == THANOS_UNSTRUCTURED) {
-    // The tie kernels work whenever the threshold value is shared by entries on both sides of
-    // the cut -- with tens of millions of fp32 scores in the residual of a wide layer that is
-    // about every second block, not a rare case: they get a full grid.
-    int hg = c < NUM_SMS * 8 ? c : NUM_SMS * 8;
     // bracket + refine, or the four radix passes, or bracket + four radix passes when it misses
     const int sg = c < NUM_SMS * 4 ? c : NUM_SMS * 4;
     // residuals beyond the L2 stream from HBM and want more loads in flight
@@ -1090,8 +1085,10 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
       thanos_stats_t* a_stats = stats;
       unsigned* a_cand = w.cand;
       unsigned a_cap = (unsigned)w.cand_cap;
+      unsigned* a_rowcnt = w.rowcnt;
+      unsigned long long* a_rowbase = w.rowbase;
       void* args[] = {&a_Wc, &a_xn, &a_c, &a_b, &a_j1, &a_bw, &a_st, &a_hist, &a_lc, &a_stats, &a_cand,
-                      &a_cap};
+                      &a_cap, &a_rowcnt, &a_rowbase};
       const void* fn = big ? reinterpret_cast<const void*>(&select_rest_kernel<4>)
                            : reinterpret_cast<const void*>(&select_rest_kernel<2>);
       if (cudaLaunchCooperativeKernel(fn, dim3((unsigned)sg2), dim3(256), args, 0, stream) !=
@@ -1099,10 +1096,6 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
         return THANOS_ERR_CUDA;
       count_launch();
     }
-    tie_count_kernel<<<hg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.rowcnt);
-    THANOS_CHECK_LAUNCH();
-    tie_scan_kernel<<<1, 1024, 0, stream>>>(c, w.st, w.rowcnt, w.rowbase);
-    THANOS_CHECK_LAUNCH();
     int mg = (int)ceil_div(c, MARK_WARPS);
     if (mg > NUM_SMS * 2) mg = NUM_SMS * 2;
     mark_block_kernel<<<mg, 32 * MARK_WARPS, 0, stream>>>(Wc, xnorm, mask, c, b, j1, Bw, w.st, w.rowbase,
