@@ -623,11 +623,11 @@ __device__ __forceinline__ void tie_scan_rows(int c, const unsigned* __restrict_
   }
 }
 
-// The passes a block may still need after its first two launches (bracket + refine, or the first
-// two radix passes): up to three more radix passes, in ONE cooperative launch with a grid barrier
-// between them.  With the threshold known on entry, which is the usual case, it runs none of
-// them, so a block step carries one nearly idle launch instead of three.  Last it finds out
-// whether the order of tied entries can matter to this block's mask at all, and ranks them if so.
+// Everything a block's selection needs after its pass over the residual, in ONE cooperative launch
+// with a grid barrier between the steps: the refine pass over the copied keys (the usual case), or
+// up to four radix passes (three after a first radix pass, four after a bracket that missed).
+// Last it finds out whether the order of tied entries can matter to this block's mask at all,
+// and ranks them if so.
 template <int BR_UNROLL>
 __global__ void __launch_bounds__(256)
 select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm, int c, int b,
@@ -636,7 +636,7 @@ select_rest_kernel(const float* __restrict__ Wc, const float* __restrict__ xnorm
                    unsigned* __restrict__ cand, unsigned cand_cap,
                    unsigned* __restrict__ rowcnt, unsigned long long* __restrict__ rowbase) {
   cooperative_groups::grid_group grid = cooperative_groups::this_grid();
-  for (int it = 0; it < 3; ++it) {
+  for (int it = 0; it < 4; ++it) {
     // the phase only changes between two grid barriers, so every CTA reads the same value
     if (*reinterpret_cast<volatile int*>(&st->phase) == PH_DONE) break;
     select_pass_body<BR_UNROLL>(Wc, xnorm, c, b, j1, st, hist, nullptr, list_counts, 0, stats, cand,
@@ -1061,21 +1061,19 @@ thanos_status_t block_step(float* Wc, uint8_t* mask, int c, int b, const float* 
     // residuals beyond the L2 stream from HBM and want more loads in flight
     const bool big = (size_t)c * (size_t)(b - j1) * sizeof(float) > ((size_t)96 << 20);
     const int sg2 = sg < NUM_SMS * 2 ? sg : NUM_SMS * 2;
-    for (int pass = 0; pass < 2; ++pass) {
-      // the second pass usually looks at the copied keys only
-      const int sgp = pass == 0 ? sg : sg2;
-      if (big)
-        select_pass_kernel<4><<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
-                                                      w.list_counts, pass == 0 ? 1 : 0, stats,
-                                                      w.cand, (unsigned)w.cand_cap);
-      else
-        select_pass_kernel<2><<<sgp, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
-                                                      w.list_counts, pass == 0 ? 1 : 0, stats,
-                                                      w.cand, (unsigned)w.cand_cap);
-      THANOS_CHECK_LAUNCH();
-    }
+    // the pass over the residual (bracket, or the first radix pass)
+    if (big)
+      select_pass_kernel<4><<<sg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                    w.list_counts, 1, stats, w.cand,
+                                                    (unsigned)w.cand_cap);
+    else
+      select_pass_kernel<2><<<sg, 256, 0, stream>>>(Wc, xnorm, c, b, j1, w.st, w.hist, r_ext,
+                                                    w.list_counts, 1, stats, w.cand,
+                                                    (unsigned)w.cand_cap);
+    THANOS_CHECK_LAUNCH();
     {
-      // whatever is left of a radix route, behind grid barriers (sg2 <= 2 CTAs per SM: co-resident)
+      // everything else behind grid barriers in one launch (sg2 <= 2 CTAs per SM: co-resident):
+      // the refine pass over the copied keys, or what is left of a radix route, then the ties
       const float* a_Wc = Wc;
       const float* a_xn = xnorm;
       int a_c = c, a_b = b, a_j1 = j1, a_bw = Bw;
