@@ -36,8 +36,10 @@ namespace {
 //            (512 bins of 128 values) and copies them out (about 1 in 130); a second, short pass
 //            over the copied keys resolves the 512 values of the hit bin;
 //   radix    four passes over 8, 8, 8 and 7 key bits (first block, or when the window misses).
-// One kernel, launched five times per block, does whichever pass the sweep state asks for; the
-// last CTA to finish a pass reads the histogram, decides and sets the next phase.
+// One pass body does whichever pass the sweep state asks for; the last CTA to finish a pass reads
+// the histogram, decides and sets the next phase.  Per block it runs once as a kernel of its own
+// (the pass over the residual) and then inside one cooperative launch, behind grid barriers, as
+// often as the route still needs.
 constexpr int HIST_BINS = 512;
 constexpr int RADIX_BINS = 256;
 constexpr int RADIX_REPL = 8;           // shared-memory copies of a radix histogram (by lane & 7)
