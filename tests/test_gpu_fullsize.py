@@ -314,6 +314,25 @@ def _late_block_literal(T, W, U, xn, H32, lam, mode_nm, B, j1, rows):
     assert torch.equal(Wc[:, :j1], W.float()[:, :j1])
 
 
+@pytest.mark.parametrize("b", [8200, 11008])
+def test_factor_identity_on_grouped_panels_and_cta_pairs(T, b):
+    """Widths whose factorisation runs its large products on CTA pairs (256 x 256 tiles) with the
+    panels in groups of four: 11008 (the benchmark's widest layer: 86 panels = 21 groups and two
+    left over) and 8200 (a ragged last panel of 8 columns, ragged 256-tiles in every product).
+    U is upper-triangular and U H_d U^T = I on sampled rows in float64."""
+    Xd = WL.make_activations(2 * b, b, "bf16", "student_t4", 0.005, 0, 50.0, 5, 1, device=DEV)
+    H = _hessian(T, Xd)
+    del Xd
+    U, xn = T.prepare_inverse(H, 0.01)
+    assert bool((torch.tril(U, -1) == 0).all()) and bool(torch.isfinite(U).all())
+    H32, U32 = H.cpu(), U.cpu()
+    lam = 0.01 * float(np.mean(np.diag(H32.numpy()).astype(np.float64)))
+    err = _factor_identity_error(U32, H32, lam, [0, 1, b // 2 + 3, b - 130, b - 1])
+    print("max |U H_d U^T - I| on sampled rows, b = %d: %.2e" % (b, err))
+    assert err <= 1e-4
+    assert np.allclose(_np64(xn), O.feature_norms(_np64(H)), rtol=1e-6)
+
+
 def test_llama3_8b_down_projection_width(T):
     """b = 14336 (the down projection of the LLaMA-3-8B-shaped set), 4:8, B = 256, 256 rows:
     n:m pattern and exact zeros on the whole output, the factor's defining identity on sampled
