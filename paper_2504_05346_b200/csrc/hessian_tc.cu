@@ -391,7 +391,16 @@ thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld
   return THANOS_OK;
 }
 
-constexpr int SPLIT_CHUNK = 8192;  // tokens of fp32 input split per pass
+// Tokens of fp32 input split into planes per pass: as many as fit 2^28 plane bytes (a launch over a
+// longer chunk has more token slices to fill the SMs with, which narrow layers need), between 8192
+// and 65536 and a multiple of 512.
+int64_t split_chunk_tokens(int64_t b) {
+  int64_t t = ((int64_t)1 << 28) / (6 * b);
+  t = t / 512 * 512;
+  if (t < 8192) t = 8192;
+  if (t > 65536) t = 65536;
+  return t;
+}
 
 }  // namespace
 
@@ -401,7 +410,8 @@ thanos_status_t launch_hessian_tc2(float* H, int b, const __nv_bfloat16* base, i
 
 size_t hessian_tc_workspace_bytes(int64_t b, thanos_dtype_t dtype) {
   size_t w = 256;  // status word
-  if (dtype == THANOS_F32) w += round_up((size_t)3 * SPLIT_CHUNK * b * sizeof(__nv_bfloat16), 256);
+  if (dtype == THANOS_F32)
+    w += round_up((size_t)3 * (size_t)split_chunk_tokens(b) * b * sizeof(__nv_bfloat16), 256);
   return w;
 }
 
@@ -430,8 +440,9 @@ thanos_status_t hessian_accumulate_tc(float* H, int64_t b, const void* X, thanos
     return THANOS_OK;
   }
   __nv_bfloat16* planes = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + 256);
-  for (int64_t t0 = 0; t0 < n_tok; t0 += SPLIT_CHUNK) {
-    int n = (int)(n_tok - t0 < SPLIT_CHUNK ? n_tok - t0 : SPLIT_CHUNK);
+  const int64_t chunk = split_chunk_tokens(b);
+  for (int64_t t0 = 0; t0 < n_tok; t0 += chunk) {
+    int n = (int)(n_tok - t0 < chunk ? n_tok - t0 : chunk);
     split_planes_kernel<<<NUM_SMS * 8, 256, 0, stream>>>(static_cast<const float*>(X) + t0 * ldx, ldx,
                                                      n, (int)b, planes);
     THANOS_CHECK_LAUNCH();
