@@ -9,8 +9,8 @@
 //               at the end of a unit 2*acc is added to H[i, j] and to the mirror H[j, i].
 // TMEM: two 128 x 256 fp32 accumulators (all 512 columns), so draining overlaps the next MMAs.
 // Only tiles that touch the upper triangle are computed.  fp32 inputs are first split into
-// three bf16 planes (x = h + m + l); the six significant plane products hh, hm, mh, hl, lh, mm
-// run through the same pipeline as extra contraction steps.
+// three bf16 planes (x = h + m + l); a stage then holds all three planes of 32 tokens, and the six
+// significant plane products hh, hm, mh, hl, lh, mm are issued from it.
 //
 // Every wait is bounded: on expiry the CTA raises an abort flag, records THANOS_ERR_TIMEOUT in
 // the status word, drains, frees its TMEM and returns.
@@ -22,14 +22,25 @@ namespace {
 
 constexpr int TM = 128;           // tile rows (features i)
 constexpr int TN = 256;           // tile columns (features j)
-constexpr int BK = 64;            // tokens per pipeline stage
-constexpr int STAGES = 4;
-constexpr int FLUSH_STAGES = 8;   // TMEM accumulator drained every 8 stages = 512 tokens
-constexpr int BOX_BYTES = 64 * BK * 2;             // one 64-feature x 64-token bf16 box
-constexpr int STAGE_BYTES = 6 * BOX_BYTES;         // 4 boxes for the j block, 2 for the i block
-constexpr int A_OFFSET = 4 * BOX_BYTES;
 constexpr int NTHREADS = 320;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+// Pipeline geometry.  One plane (bf16 input): 64 tokens per stage, 4 boxes of 64 features for the j
+// block and 2 for the i block (48 KB), four stages, the accumulator drained every 8 stages = 512
+// tokens = 32 MMAs.  Three planes (split fp32 input): all three planes of both blocks for 32
+// tokens per stage (72 KB, three stages), from which the six plane products are issued -- every
+// plane is loaded once per token step, not once per product --, drained every 3 stages = 96
+// tokens = 36 MMAs.
+template <bool P3>
+struct Geo {
+  static constexpr int BK = P3 ? 32 : 64;
+  static constexpr int STAGES = P3 ? 3 : 4;
+  static constexpr int FLUSH_STAGES = P3 ? 3 : 8;
+  static constexpr int BOX_BYTES = 64 * BK * 2;            // one 64-feature x BK-token bf16 box
+  static constexpr int PLANE_BYTES = 6 * BOX_BYTES;        // 4 boxes of the j block, 2 of the i block
+  static constexpr int A_OFFSET = 4 * BOX_BYTES;
+  static constexpr int STAGE_BYTES = (P3 ? 3 : 1) * PLANE_BYTES;
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
 
 struct Params {
   float* H;
@@ -50,10 +61,10 @@ using namespace tc;
 // Shared-memory matrix descriptor for an MN-major bf16 operand stored as 64-feature x 64-token
 // boxes with the 128-byte swizzle: a token is one 128-byte row, 8 tokens form a 1024-byte
 // swizzle atom (stride offset), the next 64 features live one box further (leading offset).
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t box_bytes) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((uint32_t)BOX_BYTES >> 4) << 16;  // leading-dimension byte offset
+  d |= (uint64_t)(box_bytes >> 4) << 16;            // leading-dimension byte offset
   d |= (uint64_t)(1024u >> 4) << 32;                // stride-dimension byte offset
   d |= (uint64_t)1 << 46;                           // descriptor version for sm_100
   d |= (uint64_t)2 << 61;                           // 128-byte swizzle
@@ -78,7 +89,7 @@ struct Unit {
   bool diag;
 };
 
-__device__ __forceinline__ Unit decode_unit(const Params& p, int u) {
+__device__ __forceinline__ Unit decode_unit(const Params& p, int u, int bk) {
   Unit r;
   int tile = u % p.n_tiles;
   int slice = u / p.n_tiles;
@@ -95,18 +106,23 @@ __device__ __forceinline__ Unit decode_unit(const Params& p, int u) {
   r.t0 = slice * p.slice_tokens;
   int t1 = r.t0 + p.slice_tokens;
   if (t1 > p.n_tok) t1 = p.n_tok;
-  r.nst = (t1 - r.t0 + BK - 1) / BK;
+  r.nst = (t1 - r.t0 + bk - 1) / bk;
   if (r.nst < 0) r.nst = 0;
   return r;
 }
 
+template <bool P3>
 __global__ void __launch_bounds__(NTHREADS, 1)
 hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
+  using G = Geo<P3>;
+  constexpr int BK = G::BK, STAGES = G::STAGES, FLUSH_STAGES = G::FLUSH_STAGES;
+  constexpr int BOX_BYTES = G::BOX_BYTES, STAGE_BYTES = G::STAGE_BYTES, A_OFFSET = G::A_OFFSET;
+  constexpr int PLANE_BYTES = G::PLANE_BYTES;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
-  // bars[0..3] full, [4..7] empty, [8..9] tmem full, [10..11] tmem empty
+  // bars[0..3] full, [4..7] empty, [8..9] tmem full, [10..11] tmem empty (STAGES <= 4)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 13);
 
@@ -150,26 +166,31 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     uint32_t phase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const Unit un = decode_unit(p, u);
-      const int total = un.nst * p.n_combo;
+      const Unit un = decode_unit(p, u, BK);
+      const int total = P3 ? un.nst : un.nst * p.n_combo;
       for (int kk = 0; kk < total && ok; ++kk) {
-        const int combo = kk / un.nst;
+        const int combo = P3 ? 0 : kk / un.nst;
         const int ks = kk - combo * un.nst;
         const int pa = p.plane_a[combo], pb = p.plane_b[combo];
-        const bool shortcut = un.diag && pa == pb;
+        // on a diagonal tile the i block is one half of the j block (of the same plane)
+        const bool shortcut = un.diag && (P3 || pa == pb);
         ok = mbar_wait(empty_bar(s), phase ^ 1u, abort_flag);
         if (ok && lane == 0) {
           const uint32_t dst = smem_base + (uint32_t)s * STAGE_BYTES;
           const int y = un.t0 + ks * BK;
-          mbar_expect_tx(full_bar(s), shortcut ? 4 * BOX_BYTES : 6 * BOX_BYTES);
+          mbar_expect_tx(full_bar(s), (P3 ? 3 : 1) * (shortcut ? 4 * BOX_BYTES : 6 * BOX_BYTES));
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            tma_load_3d(dst + i * BOX_BYTES, &tmap, full_bar(s), un.J * TN + 64 * i, y, pb);
-          if (!shortcut) {
+          for (int pl = 0; pl < (P3 ? 3 : 1); ++pl) {
+            const uint32_t d0 = dst + (uint32_t)pl * PLANE_BYTES;
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
-              tma_load_3d(dst + A_OFFSET + i * BOX_BYTES, &tmap, full_bar(s), un.I * TM + 64 * i,
-                          y, pa);
+            for (int i = 0; i < 4; ++i)
+              tma_load_3d(d0 + i * BOX_BYTES, &tmap, full_bar(s), un.J * TN + 64 * i, y, P3 ? pl : pb);
+            if (!shortcut) {
+#pragma unroll
+              for (int i = 0; i < 2; ++i)
+                tma_load_3d(d0 + A_OFFSET + i * BOX_BYTES, &tmap, full_bar(s), un.I * TM + 64 * i, y,
+                            P3 ? pl : pa);
+            }
           }
         }
         __syncwarp();
@@ -190,26 +211,33 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     uint32_t phase = 0, tphase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const Unit un = decode_unit(p, u);
-      const int total = un.nst * p.n_combo;
+      const Unit un = decode_unit(p, u, BK);
+      const int total = P3 ? un.nst : un.nst * p.n_combo;
       for (int g0 = 0; g0 < total && ok; g0 += FLUSH_STAGES) {
         const int g1 = g0 + FLUSH_STAGES < total ? g0 + FLUSH_STAGES : total;
         ok = mbar_wait(tempty_bar(q), tphase ^ 1u, abort_flag);
         tc_fence_after();
         for (int kk = g0; kk < g1 && ok; ++kk) {
-          const int combo = kk / un.nst;
-          const bool shortcut = un.diag && p.plane_a[combo] == p.plane_b[combo];
+          const int combo = P3 ? 0 : kk / un.nst;
           ok = mbar_wait(full_bar(s), phase, abort_flag);
           tc_fence_after();
           if (ok && lane == 0) {
-            const uint32_t sb = smem_base + (uint32_t)s * STAGE_BYTES;
-            const uint32_t sa = shortcut ? sb + (uint32_t)(un.I & 1) * 2 * BOX_BYTES : sb + A_OFFSET;
+            const uint32_t stage = smem_base + (uint32_t)s * STAGE_BYTES;
 #pragma unroll
-            for (int k4 = 0; k4 < BK / 16; ++k4) {
-              const uint64_t adesc = make_desc(sa + k4 * 2048);
-              const uint64_t bdesc = make_desc(sb + k4 * 2048);
-              tc_mma_bf16(tmem_base + (uint32_t)q * TN, adesc, bdesc, idesc,
-                          (kk > g0 || k4 > 0) ? 1u : 0u);
+            for (int cb = 0; cb < (P3 ? 6 : 1); ++cb) {
+              const int pa = p.plane_a[P3 ? cb : combo], pb = p.plane_b[P3 ? cb : combo];
+              const bool shortcut = un.diag && (P3 || pa == pb);
+              const uint32_t sb = stage + (P3 ? (uint32_t)pb * PLANE_BYTES : 0u);
+              const uint32_t pa_base = stage + (P3 ? (uint32_t)pa * PLANE_BYTES : 0u);
+              const uint32_t sa =
+                  shortcut ? pa_base + (uint32_t)(un.I & 1) * 2 * BOX_BYTES : pa_base + A_OFFSET;
+#pragma unroll
+              for (int k4 = 0; k4 < BK / 16; ++k4) {
+                const uint64_t adesc = make_desc(sa + k4 * 2048, BOX_BYTES);
+                const uint64_t bdesc = make_desc(sb + k4 * 2048, BOX_BYTES);
+                tc_mma_bf16(tmem_base + (uint32_t)q * TN, adesc, bdesc, idesc,
+                            (kk > g0 || cb > 0 || k4 > 0) ? 1u : 0u);
+              }
             }
             tc_commit(empty_bar(s));
           }
@@ -236,8 +264,8 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     uint32_t tphase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const Unit un = decode_unit(p, u);
-      const int total = un.nst * p.n_combo;
+      const Unit un = decode_unit(p, u, BK);
+      const int total = P3 ? un.nst : un.nst * p.n_combo;
       float acc[128];
 #pragma unroll
       for (int k = 0; k < 128; ++k) acc[k] = 0.f;
@@ -300,23 +328,33 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
   if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, (int)THANOS_ERR_TIMEOUT);
 }
 
-// x = h + m + l with three bf16 planes [3][n][b] (fp32 has 24 significant bits, 3 x 8)
+// x = h + m + l with three bf16 planes [3][n][b] (fp32 has 24 significant bits, 3 x 8); four
+// consecutive features per thread (b and ldx are multiples of 8)
 __global__ void split_planes_kernel(const float* __restrict__ X, int64_t ldx, int n, int b,
                                     __nv_bfloat16* __restrict__ planes) {
+  const int b4 = b >> 2;
+  const int64_t total4 = (int64_t)n * b4;
   const int64_t total = (int64_t)n * b;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
-    int64_t t = e / b;
-    int j = (int)(e - t * b);
-    float x = X[t * ldx + j];
-    __nv_bfloat16 hh = __float2bfloat16_rn(x);
-    float r1 = x - __bfloat162float(hh);
-    __nv_bfloat16 mm = __float2bfloat16_rn(r1);
-    float r2 = r1 - __bfloat162float(mm);
-    __nv_bfloat16 ll = __float2bfloat16_rn(r2);
-    planes[e] = hh;
-    planes[total + e] = mm;
-    planes[2 * total + e] = ll;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total4; e += stride) {
+    const int64_t t = e / b4;
+    const int j = 4 * (int)(e - t * b4);
+    const float4 xv = *reinterpret_cast<const float4*>(X + t * ldx + j);
+    float x[4] = {xv.x, xv.y, xv.z, xv.w};
+    const int64_t o = t * b + j;
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      __nv_bfloat16 hb[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        hb[k] = __float2bfloat16_rn(x[k]);
+        x[k] -= __bfloat162float(hb[k]);
+      }
+      uint2 pk;
+      pk.x = (uint32_t)__bfloat16_as_ushort(hb[0]) | ((uint32_t)__bfloat16_as_ushort(hb[1]) << 16);
+      pk.y = (uint32_t)__bfloat16_as_ushort(hb[2]) | ((uint32_t)__bfloat16_as_ushort(hb[3]) << 16);
+      *reinterpret_cast<uint2*>(planes + (int64_t)pl * total + o) = pk;
+    }
   }
 }
 
@@ -328,6 +366,9 @@ thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld
   CUtensorMap tmap;
   cuuint64_t gdim[3] = {(cuuint64_t)b, (cuuint64_t)n_tok, (cuuint64_t)planes};
   cuuint64_t gstr[2] = {(cuuint64_t)ld_elems * 2, (cuuint64_t)plane_stride_elems * 2};
+  const bool p3 = planes == 3;
+  const int BK = p3 ? Geo<true>::BK : Geo<false>::BK;
+  const int FLUSH_STAGES = p3 ? Geo<true>::FLUSH_STAGES : Geo<false>::FLUSH_STAGES;
   cuuint32_t box[3] = {64, (cuuint32_t)BK, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(base), gdim, gstr,
@@ -382,11 +423,15 @@ thanos_status_t launch_tc(float* H, int b, const __nv_bfloat16* base, int64_t ld
   }
   long long units = (long long)p.n_tiles * p.n_slices;
   int grid = (int)(units < G ? units : G);
-  {
+  if (p3) {
     static std::atomic<unsigned long long> done{0};
-    THANOS_CUDA(ensure_max_dyn_smem(hessian_tc_kernel, (int)SMEM_BYTES, done));
+    THANOS_CUDA(ensure_max_dyn_smem(hessian_tc_kernel<true>, (int)Geo<true>::SMEM_BYTES, done));
+    hessian_tc_kernel<true><<<grid, NTHREADS, Geo<true>::SMEM_BYTES, stream>>>(tmap, p);
+  } else {
+    static std::atomic<unsigned long long> done{0};
+    THANOS_CUDA(ensure_max_dyn_smem(hessian_tc_kernel<false>, (int)Geo<false>::SMEM_BYTES, done));
+    hessian_tc_kernel<false><<<grid, NTHREADS, Geo<false>::SMEM_BYTES, stream>>>(tmap, p);
   }
-  hessian_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(tmap, p);
   THANOS_CHECK_LAUNCH();
   return THANOS_OK;
 }
