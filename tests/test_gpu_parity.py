@@ -71,11 +71,14 @@ def test_hessian_strided_input_and_empty_chunk(T):
     assert PU.rel_fro(_np64(H), Ho) <= PU.TOL_H
 
 
-@pytest.mark.parametrize("b,n_tok", [(4096, 32768), (11008, 12345)])
-def test_hessian_bench_shape_sampled(T, b, n_tok):
-    """The benchmark's layer widths with long bf16 chunks (CTA-pair kernel, several token slices,
-    a ragged token tail): sampled entries against a float64 dot product."""
-    Xd = WL.make_activations(n_tok, b, "bf16", "student_t4", 0.005, 0, 50.0, 2, 0, device=DEV)
+@pytest.mark.parametrize("b,n_tok,dtype", [(4096, 32768, "bf16"), (11008, 12345, "bf16"),
+                                           (768, 70001 // 8 * 8, "f32"), (3072, 20000, "f32")])
+def test_hessian_bench_shape_sampled(T, b, n_tok, dtype):
+    """The benchmark's layer widths with long chunks (bf16: CTA-pair kernel, several token slices,
+    a ragged token tail; fp32: the widths of the OPT-125M-shaped set, more tokens than one pass of
+    the split into planes takes, stages that hold all three planes): sampled entries against a
+    float64 dot product."""
+    Xd = WL.make_activations(n_tok, b, dtype, "student_t4", 0.005, 0, 50.0, 2, 0, device=DEV)
     H = torch.zeros((b, b), dtype=torch.float32, device=DEV)
     T.hessian_accumulate(H, Xd)
     torch.cuda.synchronize()
